@@ -1,0 +1,372 @@
+#!/usr/bin/env python
+"""Benchmark of the dual-precision linear-layer path on B200.
+
+One "step" is one pass of the decode hot path over the Llama-7B-shaped workload: for every
+token count M in {1, 8, 32} and for both modes (fast = persistent plane only, full =
+persistent + residual planes), the four linears of a decoder layer (QKV, O, gate+up, down)
+are run over `--copies` distinct weight copies, so that between two reads of the same plane
+several times the L2 capacity has streamed by.  Each (M, mode) pair is one CUDA graph (the
+paper pre-captures one graph per mode and batch size and picks one per forward pass).
+
+The JSON line reports
+  value     decode throughput in algorithmic GB/s (weights + activations + outputs, the
+            bytes the method has to move) with everything resident in HBM,
+  e2e       the same pass through the public binding with the activations coming from and
+            the outputs going back to pinned host memory inside the timed region,
+  roofline  the same bytes against the measured HBM copy bandwidth,
+  cpu_baseline  the CPU oracle timed on a bounded sample of the same workload,
+plus per-(M, mode) figures and the other measured rows of the path under "detail".
+
+`--impl reference` times the CPU oracle alone (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "decode linear-layer HBM GB/s (algorithmic bytes / time), Llama-7B-shaped linears, M in {1,8,32}, both modes"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--copies", type=int, default=32, help="distinct weight copies per linear (L2 rotation)")
+    ap.add_argument("--skip-detail", action="store_true", help="skip the extra rows (split, prefill, MoE)")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="time budget of the CPU oracle sample")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = ROOT / "MEASURED_PEAKS.json"
+    if path.exists():
+        d = json.loads(path.read_text())
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])), mx.append(float(r[1])), pw.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+# --------------------------------------------------------------------------------------------
+
+def linear_bytes(mode_full: bool, m: int, n: int, k: int) -> int:
+    return n * k * (2 if mode_full else 1) + 2 * m * k + 2 * m * n
+
+
+def oracle_sample(budget_s: float, threads: int):
+    """Runs the oracle as it stands on Llama-7B-shaped linears at M=1, both modes, smallest
+    layer first, until the time budget is used.  Returns (GB/s, description, seconds)."""
+    import numpy as np
+    import oracle
+    from paper_2609_34380_b200 import workloads
+
+    order = ["o", "down", "qkv", "gate_up"]
+    done, total_bytes, total_s = [], 0, 0.0
+    for name in order:
+        n, k = workloads.LLAMA7B[name]
+        if done and total_s > budget_s * 0.6:
+            break
+        rng = np.random.default_rng(2001)
+        w = (rng.standard_normal((n, k), dtype=np.float32) * 0.02).astype(np.float16)
+        x = rng.standard_normal((1, k), dtype=np.float32).astype(np.float16)
+        p, r, enc = oracle.split(w, oracle.ENC_AUTO)
+        for mode in (oracle.MODE_FAST, oracle.MODE_FULL):
+            t0 = time.perf_counter()
+            oracle.linear(mode, enc, x, p, r if mode else None, threads=threads)
+            total_s += time.perf_counter() - t0
+            total_bytes += linear_bytes(bool(mode), 1, n, k)
+        done.append(name)
+    gbs = total_bytes / total_s / 1e9
+    return gbs, f"oracle.linear (FP64, {threads} threads) on Llama-7B linears {done} at M=1, fast+full", total_s
+
+
+def run_reference(args, rank: int):
+    if rank != 0:
+        return
+    threads = os.cpu_count() or 1
+    budget = max(2.0, min(args.cpu_seconds, 240.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(budget, threads)
+    vals, secs, sample = [], [], ""
+    for _ in range(args.steps):
+        v, sample, s = oracle_sample(budget, threads)
+        vals.append(v)
+        secs.append(s)
+    value = sum(vals) / len(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config 2 sample: " + sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------
+
+def run_ours(args, rank: int, local_rank: int, world: int):
+    import torch
+    import paper_2609_34380_b200 as dps
+    from paper_2609_34380_b200 import workloads
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+    peaks = measured_peaks()
+
+    layers = list(workloads.LLAMA7B.items())
+    Ms = list(workloads.DECODE_M)
+    modes = [dps.DPS_MODE_FAST, dps.DPS_MODE_FULL]
+    copies = args.copies
+
+    # ---- resident model state: nested planes for every copy of every linear -------------------
+    planes = {}
+    for li, (name, (n, k)) in enumerate(layers):
+        P = torch.empty((copies, n, k), dtype=torch.uint8, device=dev)
+        R = torch.empty((copies, n, k), dtype=torch.uint8, device=dev)
+        enc_used = None
+        for c in range(copies):
+            w = workloads.weights(n, k, 2001 + li + 100 * c + 10000 * rank, device=dev)
+            _, _, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO, P[c], R[c])
+            enc_used = enc if enc_used is None else enc_used
+            assert enc == enc_used
+            del w
+        planes[name] = (P, R, enc_used)
+    xs = {(name, M): workloads.activations(M, k, 2011 + li, device=dev)
+          for li, (name, (n, k)) in enumerate(layers) for M in Ms}
+    ys = {(name, M): torch.empty((M, n), dtype=torch.float16, device=dev)
+          for (name, (n, k)) in layers for M in Ms}
+
+    def enqueue(M, mode):
+        for c in range(copies):
+            for name, (n, k) in layers:
+                P, R, enc = planes[name]
+                dps.dps_linear(mode, enc, xs[(name, M)], P[c], R[c] if mode else None, ys[(name, M)])
+
+    bytes_of = {(M, mode): copies * sum(linear_bytes(bool(mode), M, n, k) for _, (n, k) in layers)
+                for M in Ms for mode in modes}
+    flops_of = {(M, mode): copies * sum(2 * M * n * k for _, (n, k) in layers) for M in Ms for mode in modes}
+    step_bytes = sum(bytes_of.values())
+
+    # ---- one CUDA graph per (M, mode) ----------------------------------------------------------
+    stream = torch.cuda.Stream(device=dev)
+    graphs, launches_per_graph = {}, {}
+    with torch.cuda.stream(stream):
+        for key in bytes_of:
+            enqueue(*key)                       # eager warm-up (also performs the library's one-time set-up)
+        stream.synchronize()
+        for key in bytes_of:
+            before = dps.dps_launch_count()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                enqueue(*key)
+            graphs[key] = g
+            launches_per_graph[key] = dps.dps_launch_count() - before
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step(events=None):
+        for i, key in enumerate(graphs):
+            if events is not None:
+                events[i].record(stream)
+            graphs[key].replay()
+        if events is not None:
+            events[len(graphs)].record(stream)
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            step()
+        barrier()
+        sampler = ClockSampler(local_rank)
+        sampler.start()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(graphs) + 1)] for _ in range(args.steps)]
+        barrier()
+        for s in range(args.steps):
+            step(ev[s])
+        barrier()
+        clocks = sampler.stop()
+    total_ms = ev[0][0].elapsed_time(ev[-1][len(graphs)])
+    per_key_ms = {key: statistics.median(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(args.steps))
+                  for i, key in enumerate(graphs)}
+    launches = args.steps * sum(launches_per_graph.values())
+
+    # ---- end to end through the binding: activations from pinned host, outputs back ------------
+    xs_host = {k_: v.cpu().pin_memory() for k_, v in xs.items()}
+    ys_host = {k_: torch.empty_like(v, device="cpu").pin_memory() for k_, v in ys.items()}
+    h2d = copies * 0 + sum(v.numel() * 2 for v in xs_host.values()) * len(modes)
+    d2h = sum(v.numel() * 2 for v in ys_host.values()) * len(modes)
+
+    def e2e_step():
+        for M in Ms:
+            for mode in modes:
+                for name, _ in layers:
+                    xs[(name, M)].copy_(xs_host[(name, M)], non_blocking=True)
+                enqueue(M, mode)
+                for name, _ in layers:
+                    ys_host[(name, M)].copy_(ys[(name, M)], non_blocking=True)
+        stream.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e2e_steps = max(2, min(args.steps, 5))
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    # ---- max over ranks --------------------------------------------------------------------------
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = total_ms / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * step_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9
+
+    per_rank_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    detail = {"per_M_mode": {}}
+    for (M, mode), ms in per_key_ms.items():
+        b = bytes_of[(M, mode)]
+        t_roof = max(b / (peaks["hbm_gbs"] * 1e9), flops_of[(M, mode)] / (peaks["bf16_tflops"] * 1e12))
+        detail["per_M_mode"][f"M{M}_{'full' if mode else 'fast'}"] = {
+            "ms": ms, "GB/s": b / (ms * 1e-3) / 1e9, "frac_of_measured_hbm": (b / (ms * 1e-3) / 1e9) / peaks["hbm_gbs"],
+            "frac_of_nominal_8TBs": (b / (ms * 1e-3) / 1e9) / NOMINAL_HBM_GBS, "frac_of_roofline": t_roof / (ms * 1e-3),
+            "us_per_layer_set": 1e3 * ms / copies}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
+        "config": {"workload": "config 2: Llama-7B-shaped decoder-layer linears (QKV 12288x4096, O 4096x4096, "
+                               "gate+up 22016x4096, down 4096x11008), M in {1,8,32}, fast+full mode",
+                   "weight_copies": copies, "l2": f"inputs larger than L2: {copies} distinct copies "
+                   f"({copies * 202.4 / 1e3:.1f} GB of persistent planes) streamed between reuses",
+                   "graphs": "one CUDA graph per (M, mode)", "multi_gpu": "replicas only"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "achieved": per_rank_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": per_rank_gbs / peaks["hbm_gbs"], "traffic": None,
+                     "peak_source": f"{peaks['source']} (copy bandwidth)",
+                     "frac_of_nominal_8TBs": per_rank_gbs / NOMINAL_HBM_GBS,
+                     "kernel": "dense linear kernels, all launches of the step",
+                     "bytes_per_launch": step_bytes * args.steps / launches,
+                     "us_per_launch": 1e3 * total_ms / launches},
+        "detail": detail,
+    }
+    if rank == 0:
+        threads = os.cpu_count() or 1
+        if world == 1:
+            gbs, sample, secs = oracle_sample(args.cpu_seconds, threads)
+            line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                                    "seconds": secs}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

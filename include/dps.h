@@ -1,0 +1,149 @@
+/*
+ * libdps -- dual-precision (fast / full mode) linear layers computed directly from
+ * nested FP8 + residual weight planes, for NVIDIA B200 (sm_100a).
+ *
+ * The operations follow the DPS paper's statement of the problem:
+ *   - an FP16 model is split into an FP8 model kept in the persistent region and a
+ *     residual model kept in the shared region (section "Mapper: Semi-Unified Memory
+ *     Abstraction", paragraph "Persistent Region");
+ *   - in full mode the executor combines both tensors to reconstruct the original FP16
+ *     values during computation; in fast mode only the FP8 tensor is used and the
+ *     residual is not accessed, because its memory may be holding KV-cache data
+ *     (section "Scheduler: Dual-Precision Execution", paragraph "Overall concept");
+ *   - the encoding (E4M3 or E5M2) is chosen per layer at load time from weight
+ *     statistics, and the kernels serve dense and MoE (grouped) layers (same section,
+ *     paragraph "Dual-mode serving (DPS) with asymmetric switching");
+ *   - every layer of one forward pass runs in the same mode and two CUDA graphs are
+ *     captured per batch size (paragraph "Granularity of the precision switch").
+ *
+ * Conventions (all entry points):
+ *   - W[N][K] is a linear layer's weight, N outputs by K inputs, row-major with K
+ *     contiguous; y[M][N] = x[M][K] * W^T.  x and y are IEEE binary16, row-major.
+ *   - The persistent plane P and the residual plane R are SEPARATE allocations of N*K
+ *     bytes each, index-for-index identical to W.
+ *   - Pointers are DEVICE pointers unless a parameter says "host".  The caller owns
+ *     every buffer; the library never allocates or frees device memory.
+ *   - cuda_stream is a cudaStream_t passed as void* (NULL = the default stream).  Work
+ *     is enqueued on it and, except where stated, the call returns without
+ *     synchronising, so calls can be captured into CUDA graphs.
+ *   - Every device base pointer must be 16-byte aligned; K must be a multiple of 16 and
+ *     N a multiple of 8.  Violations return DPS_ERR_ALIGN / DPS_ERR_SHAPE.
+ *   - The return value reports host-detectable errors only; on error nothing has been
+ *     enqueued.  Data-dependent problems found on the device (an expert or token index
+ *     out of range) set a per-device status word: the offending row is skipped, its
+ *     output row is left untouched, and dps_stream_status() reports DPS_ERR_DATA.
+ *   - No exception crosses this boundary.  Calls on distinct streams are thread-safe.
+ */
+#ifndef DPS_H_
+#define DPS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DPS_API __attribute__((visibility("default")))
+#else
+#define DPS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DPS_OK = 0,
+    DPS_ERR_NULL = 1,        /* a required pointer is NULL */
+    DPS_ERR_SHAPE = 2,       /* negative or unsupported size */
+    DPS_ERR_MODE = 3,        /* mode is neither FAST nor FULL */
+    DPS_ERR_ENCODING = 4,    /* encoding value not valid for this call */
+    DPS_ERR_ALIGN = 5,       /* pointer not 16-byte aligned */
+    DPS_ERR_UNSUPPORTED = 6, /* valid request this build cannot serve (e.g. wrong GPU) */
+    DPS_ERR_CUDA = 7,        /* a CUDA runtime call failed */
+    DPS_ERR_DATA = 8,        /* data-dependent: E4M3 requested for an ineligible tensor, bad index */
+    DPS_ERR_WORKSPACE = 9    /* workspace NULL, misaligned or too small */
+} dps_status;
+
+typedef enum { DPS_MODE_FAST = 0, DPS_MODE_FULL = 1 } dps_mode;
+typedef enum { DPS_ENC_AUTO = 0, DPS_ENC_E4M3 = 1, DPS_ENC_E5M2 = 2 } dps_encoding;
+
+/*
+ * Nested split (paper: "Persistent Region" paragraph).  With b the FP16 word
+ * (s = b[15], e = b[14:10], m = b[9:0]):
+ *   E5M2: P = s e[4:0] m[9:8]          R = m[7:0]
+ *   E4M3: P = s e[3:0] m[9:7]          R = 0 m[6:0]      (needs b[14] == 0 everywhere)
+ * Bits are selected, never rounded, so (P, R) rebuilds W exactly.
+ *
+ * w_fp16: device, rows*cols FP16 words.  w_persist, w_resid: device, rows*cols bytes each.
+ * enc_inout: HOST int32.  On entry DPS_ENC_AUTO, DPS_ENC_E4M3 or DPS_ENC_E5M2; on return
+ * the encoding that was used.
+ *   AUTO  -> E4M3 iff every word has b[14] == 0 and max|w| <= 1.75, else E5M2.  The
+ *            statistics pass needs its result on the host, so this variant SYNCHRONISES
+ *            the stream (splitting is load-time work).
+ *   E4M3  -> also synchronises: the tensor is checked first, and if any word has b[14] set
+ *            or would produce the byte 0x7F/0xFF the call returns DPS_ERR_DATA with both
+ *            planes untouched.
+ *   E5M2  -> always legal, never synchronises.
+ * rows*cols == 0 returns DPS_OK (AUTO then reports E4M3).  cols must be a multiple of 16.
+ */
+DPS_API dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_resid,
+                             int64_t rows, int64_t cols, int32_t* enc_inout, void* cuda_stream);
+
+/*
+ * Reconstruction (paper: "Overall concept" paragraph, full mode): the inverse of the
+ * split, W = join(P, R), bit-exact.  Bit 7 of an E4M3 residual byte is ignored.
+ * w_resid == NULL rebuilds the fast-mode weights instead (residual taken as zero).
+ * enc must be DPS_ENC_E4M3 or DPS_ENC_E5M2.  Never synchronises.
+ */
+DPS_API dps_status dps_reconstruct(const uint8_t* w_persist, const uint8_t* w_resid, void* w_fp16_out,
+                           int64_t rows, int64_t cols, int32_t enc, void* cuda_stream);
+
+/*
+ * Dense linear layer (paper: "Overall concept" paragraph).
+ *   y[M][N] (FP16) = x[M][K] (FP16) * W_eff^T, FP32 accumulation, one FP16 rounding at the
+ *   store.  FULL: W_eff = join(P, R), the original FP16 weights.  FAST: W_eff = join(P, 0);
+ *   w_resid is never dereferenced and may be NULL or point at unrelated data.
+ * enc must be E4M3 or E5M2 (the value dps_split_weights reported).  M == 0 returns DPS_OK
+ * without a launch.  Never synchronises, never allocates.  Results are deterministic: the
+ * same inputs give the same bits on every call.
+ */
+DPS_API dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w_persist,
+                      const uint8_t* w_resid, void* y, int64_t M, int64_t N, int64_t K,
+                      void* cuda_stream);
+
+/*
+ * Grouped (MoE) linear layer (paper: "Dual-mode serving" paragraph, GroupedGEMM kernels).
+ * For each row a in [0, A):
+ *   y[a][:] = x[token_of_row ? token_of_row[a] : a][:] * W_eff(expert_of_row[a])^T
+ * x: [T][K] FP16.  y: [A][N] FP16.  w_persist / w_resid: [E][N][K] bytes (w_resid may be
+ * NULL in FAST mode).  enc_per_expert: HOST array of E encodings (E4M3 or E5M2), read
+ * before the call returns.  token_of_row (may be NULL) and expert_of_row: device int32[A].
+ * workspace: device scratch of at least dps_moe_workspace_bytes(A, E) bytes, 16-byte
+ * aligned, owned by the caller; its contents are overwritten.  A row whose expert is
+ * outside [0, E) or whose token is outside [0, T) is skipped and flagged (see
+ * dps_stream_status).  A == 0 returns DPS_OK without a launch.  Never synchronises.
+ */
+DPS_API dps_status dps_moe_linear(int32_t mode, const int32_t* enc_per_expert, const void* x,
+                          const int32_t* token_of_row, const int32_t* expert_of_row,
+                          const uint8_t* w_persist, const uint8_t* w_resid, void* y,
+                          int64_t A, int64_t T, int64_t N, int64_t K, int32_t E,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Bytes of scratch dps_moe_linear needs for A rows and E experts (0 if A or E is invalid). */
+DPS_API size_t dps_moe_workspace_bytes(int64_t A, int32_t E);
+
+/*
+ * Synchronises the stream, then returns and clears the current device's status word:
+ * DPS_OK, DPS_ERR_DATA (a kernel skipped a row with a bad index) or DPS_ERR_CUDA.
+ */
+DPS_API dps_status dps_stream_status(void* cuda_stream);
+
+/* Number of kernel launches this process has enqueued through the library so far. */
+DPS_API int64_t dps_launch_count(void);
+
+DPS_API const char* dps_status_string(dps_status status);
+DPS_API int dps_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DPS_H_ */

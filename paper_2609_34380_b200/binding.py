@@ -1,0 +1,175 @@
+"""Thin ctypes binding over libdps.so: same names as the C ABI, argument marshalling only.
+
+Every computation runs inside the CUDA library.  PyTorch is used for device memory and
+streams.  If the library has not been built the import of a function fails loudly; there is
+no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+DPS_MODE_FAST, DPS_MODE_FULL = 0, 1
+DPS_ENC_AUTO, DPS_ENC_E4M3, DPS_ENC_E5M2 = 0, 1, 2
+DPS_OK = 0
+DPS_ERR_NULL, DPS_ERR_SHAPE, DPS_ERR_MODE, DPS_ERR_ENCODING, DPS_ERR_ALIGN = 1, 2, 3, 4, 5
+DPS_ERR_UNSUPPORTED, DPS_ERR_CUDA, DPS_ERR_DATA, DPS_ERR_WORKSPACE = 6, 7, 8, 9
+
+LIB_PATH = Path(__file__).resolve().parent / "libdps.so"
+
+# name -> (restype, argtypes); must list every function include/dps.h declares
+_vp, _i64, _i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
+ABI = {
+    "dps_split_weights": (ctypes.c_int, [_vp, _vp, _vp, _i64, _i64, ctypes.POINTER(_i32), _vp]),
+    "dps_reconstruct": (ctypes.c_int, [_vp, _vp, _vp, _i64, _i64, _i32, _vp]),
+    "dps_linear": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
+    "dps_moe_linear": (ctypes.c_int, [_i32, ctypes.POINTER(_i32), _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64,
+                                      _i64, _i32, _vp, ctypes.c_size_t, _vp]),
+    "dps_moe_workspace_bytes": (ctypes.c_size_t, [_i64, _i32]),
+    "dps_stream_status": (ctypes.c_int, [_vp]),
+    "dps_launch_count": (_i64, []),
+    "dps_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "dps_version": (ctypes.c_int, []),
+}
+
+_lib = None
+
+
+class DpsError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: {status_string(status)} (dps_status {status})")
+        self.status = status
+
+
+def library() -> ctypes.CDLL:
+    """Load libdps.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2609_34380_b200.build` "
+                "(there is no fallback path)")
+        lib = ctypes.CDLL(str(LIB_PATH))
+        for name, (res, args) in ABI.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return library().dps_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != DPS_OK:
+        raise DpsError(status, what)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dev(t: Optional[torch.Tensor], dtype, what: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{what} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{what} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{what} must be contiguous")
+    return t.data_ptr()
+
+
+def dps_split_weights(w_fp16: torch.Tensor, enc: int = DPS_ENC_AUTO, w_persist: Optional[torch.Tensor] = None,
+                      w_resid: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor, int]:
+    """FP16 W[rows][cols] -> (persistent plane, residual plane, encoding used)."""
+    rows, cols = w_fp16.shape
+    if w_persist is None:
+        w_persist = torch.empty((rows, cols), dtype=torch.uint8, device=w_fp16.device)
+    if w_resid is None:
+        w_resid = torch.empty((rows, cols), dtype=torch.uint8, device=w_fp16.device)
+    enc_io = _i32(int(enc))
+    st = library().dps_split_weights(_dev(w_fp16, torch.float16, "w_fp16"), _dev(w_persist, torch.uint8, "w_persist"),
+                                     _dev(w_resid, torch.uint8, "w_resid"), rows, cols, ctypes.byref(enc_io),
+                                     _stream(stream))
+    _check(st, "dps_split_weights")
+    return w_persist, w_resid, int(enc_io.value)
+
+
+def dps_reconstruct(w_persist: torch.Tensor, w_resid: Optional[torch.Tensor], enc: int,
+                    w_fp16_out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """(P, R) -> the original FP16 weights; R = None gives the fast-mode weights."""
+    rows, cols = w_persist.shape
+    if w_fp16_out is None:
+        w_fp16_out = torch.empty((rows, cols), dtype=torch.float16, device=w_persist.device)
+    st = library().dps_reconstruct(_dev(w_persist, torch.uint8, "w_persist"), _dev(w_resid, torch.uint8, "w_resid"),
+                                   _dev(w_fp16_out, torch.float16, "w_fp16_out"), rows, cols, int(enc),
+                                   _stream(stream))
+    _check(st, "dps_reconstruct")
+    return w_fp16_out
+
+
+def dps_linear(mode: int, enc: int, x: torch.Tensor, w_persist: torch.Tensor, w_resid: Optional[torch.Tensor],
+               y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """y[M][N] = x[M][K] * W_eff^T from the planes, in fast or full mode."""
+    M, K = x.shape
+    N, K2 = w_persist.shape
+    if K != K2:
+        raise ValueError(f"K mismatch: x has {K}, planes have {K2}")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=x.device)
+    st = library().dps_linear(int(mode), int(enc), _dev(x, torch.float16, "x"),
+                              _dev(w_persist, torch.uint8, "w_persist"), _dev(w_resid, torch.uint8, "w_resid"),
+                              _dev(y, torch.float16, "y"), M, N, K, _stream(stream))
+    _check(st, "dps_linear")
+    return y
+
+
+def dps_moe_workspace_bytes(A: int, E: int) -> int:
+    return int(library().dps_moe_workspace_bytes(int(A), int(E)))
+
+
+def dps_moe_linear(mode: int, enc_per_expert: Sequence[int], x: torch.Tensor, token_of_row: Optional[torch.Tensor],
+                   expert_of_row: torch.Tensor, w_persist: torch.Tensor, w_resid: Optional[torch.Tensor],
+                   y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                   stream=None) -> torch.Tensor:
+    """Grouped linear: y[a] = x[token_of_row[a]] * W_eff(expert_of_row[a])^T."""
+    E, N, K = w_persist.shape
+    T, K2 = x.shape
+    if K != K2:
+        raise ValueError(f"K mismatch: x has {K}, planes have {K2}")
+    A = expert_of_row.numel()
+    if y is None:
+        y = torch.empty((A, N), dtype=torch.float16, device=x.device)
+    if workspace is None:
+        workspace = torch.empty(max(dps_moe_workspace_bytes(A, E), 16), dtype=torch.uint8, device=x.device)
+    enc_arr = (_i32 * E)(*[int(e) for e in enc_per_expert])
+    st = library().dps_moe_linear(int(mode), enc_arr, _dev(x, torch.float16, "x"),
+                                  _dev(token_of_row, torch.int32, "token_of_row"),
+                                  _dev(expert_of_row, torch.int32, "expert_of_row"),
+                                  _dev(w_persist, torch.uint8, "w_persist"), _dev(w_resid, torch.uint8, "w_resid"),
+                                  _dev(y, torch.float16, "y"), A, T, N, K, E,
+                                  _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream))
+    _check(st, "dps_moe_linear")
+    return y
+
+
+def dps_stream_status(stream=None) -> int:
+    """Synchronise the stream; return and clear the device status word."""
+    return int(library().dps_stream_status(_stream(stream)))
+
+
+def dps_launch_count() -> int:
+    return int(library().dps_launch_count())
+
+
+def dps_version() -> int:
+    return int(library().dps_version())

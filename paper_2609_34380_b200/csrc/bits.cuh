@@ -1,0 +1,67 @@
+// Device-side bit manipulation for the nested FP16 = (persistent FP8 byte, residual byte)
+// format (paper: "Mapper: Semi-Unified Memory Abstraction", "Persistent Region" paragraph).
+//
+// Everything works on 32-bit registers that hold four plane bytes (p4 / r4, element i in
+// byte i) or two FP16 words (element 2j in the low half).  No value is ever rounded: the
+// split selects bits and the join puts them back.
+#pragma once
+#include <cuda_fp16.h>
+#include <stdint.h>
+
+namespace dps {
+
+enum : int { kEncE4M3 = 1, kEncE5M2 = 2 };
+
+// E4M3 word layout inside a 16-bit lane after zipping (p << 8 | r):
+//   bit 15 = s, bits 14:11 = e[3:0], bits 10:8 = m[9:7], bits 6:0 = m[6:0]
+// FP16 wants  bit 15 = s, bit 14 = 0, bits 13:10 = e[3:0], bits 9:0 = m.
+__device__ __forceinline__ uint32_t e4m3_zipped_to_half2(uint32_t z) {
+    return (z & 0x807F807Fu) | ((z >> 1) & 0x3F803F80u);
+}
+
+// Four persistent bytes (+ four residual bytes) -> 4 FP16 words in lo (elements 0,1) and
+// hi (elements 2,3).
+template <int ENC, bool FULL>
+__device__ __forceinline__ void join4(uint32_t p4, uint32_t r4, uint32_t& lo, uint32_t& hi) {
+    if (!FULL) r4 = 0u;
+    uint32_t zl = __byte_perm(r4, p4, 0x5140);  // r0 p0 r1 p1 (low byte first)
+    uint32_t zh = __byte_perm(r4, p4, 0x7362);  // r2 p2 r3 p3
+    if (ENC == kEncE4M3) {
+        if (FULL) {
+            zl = e4m3_zipped_to_half2(zl);
+            zh = e4m3_zipped_to_half2(zh);
+        } else {  // residual is zero: only the sign and the seven kept bits move
+            zl = (zl & 0x80008000u) | ((zl >> 1) & 0x3F803F80u);
+            zh = (zh & 0x80008000u) | ((zh >> 1) & 0x3F803F80u);
+        }
+    }
+    lo = zl;
+    hi = zh;
+}
+
+// 16 plane bytes (+16 residual bytes) -> 16 FP16 words as 8 packed registers.
+template <int ENC, bool FULL>
+__device__ __forceinline__ void join16(const uint4& p, const uint4& r, uint32_t (&h)[8]) {
+    join4<ENC, FULL>(p.x, r.x, h[0], h[1]);
+    join4<ENC, FULL>(p.y, r.y, h[2], h[3]);
+    join4<ENC, FULL>(p.z, r.z, h[4], h[5]);
+    join4<ENC, FULL>(p.w, r.w, h[6], h[7]);
+}
+
+// Four FP16 words (a = elements 0,1; b = elements 2,3) -> four persistent and four residual bytes.
+template <int ENC>
+__device__ __forceinline__ void split4(uint32_t a, uint32_t b, uint32_t& p4, uint32_t& r4) {
+    if (ENC == kEncE4M3) {
+        // move e[3:0] m[9:7] (bits 13:7) up to bits 14:8, keep the sign, keep m[6:0] in the low byte
+        a = (a & 0x80008000u) | ((a << 1) & 0x7F007F00u) | (a & 0x007F007Fu);
+        b = (b & 0x80008000u) | ((b << 1) & 0x7F007F00u) | (b & 0x007F007Fu);
+    }
+    p4 = __byte_perm(a, b, 0x7531);  // high bytes
+    r4 = __byte_perm(a, b, 0x6420);  // low bytes
+}
+
+__device__ __forceinline__ float2 h2f2(uint32_t h2) {
+    return __half22float2(*reinterpret_cast<const __half2*>(&h2));
+}
+
+}  // namespace dps

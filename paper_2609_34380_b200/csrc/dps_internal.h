@@ -1,0 +1,34 @@
+// Host-side declarations shared by the translation units of libdps (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/dps.h"
+
+namespace dps {
+
+// Every launcher enqueues on `stream`, never synchronises and returns the CUDA error of the
+// launch.  `status` is the address of the current device's status word.
+
+// max over the tensor of (word & 0x7FFF), written with atomicMax into *stat (caller zeroes it).
+cudaError_t launch_magnitude_stat(const uint16_t* w, int64_t n, unsigned* stat, cudaStream_t stream);
+cudaError_t launch_split(const uint16_t* w, uint8_t* p, uint8_t* r, int64_t n, int enc, cudaStream_t stream);
+cudaError_t launch_reconstruct(const uint8_t* p, const uint8_t* r, uint16_t* w, int64_t n, int enc,
+                               cudaStream_t stream);
+
+// Dense linear, CUDA-core path (any M; efficient for M <= 4).
+cudaError_t launch_gemv(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
+                        int64_t M, int64_t N, int64_t K, cudaStream_t stream);
+
+// Grouped linear.
+size_t moe_workspace_bytes(int64_t A, int32_t E);
+cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const int32_t* token_of_row,
+                       const int32_t* expert_of_row, const uint8_t* p, const uint8_t* r, void* y, int64_t A,
+                       int64_t T, int64_t N, int64_t K, int32_t E, void* workspace, int* status,
+                       cudaStream_t stream);
+
+void count_launch(int n = 1);
+int sm_count();
+
+}  // namespace dps

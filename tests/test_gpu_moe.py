@@ -1,0 +1,138 @@
+"""GPU parity: grouped (MoE) linear layers against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_34380_b200 as dps
+from paper_2609_34380_b200 import workloads
+from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words, y_as_f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+MODES = [dps.DPS_MODE_FAST, dps.DPS_MODE_FULL]
+
+
+def expert_planes(E, N, K, seed, mixed=True):
+    ps, rs, encs = [], [], []
+    for e in range(E):
+        w = workloads.weights(N, K, seed + e, device=DEV)
+        if mixed and e % 3 == 1:
+            w = workloads.with_outlier(w)
+        p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+        ps.append(p), rs.append(r), encs.append(enc)
+    return torch.stack(ps), torch.stack(rs), encs
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("E,N,K,T", [(4, 264, 528, 10), (8, 520, 1040, 96), (3, 136, 4112, 33)])
+def test_top2_routing_small(mode, E, N, K, T):
+    p, r, encs = expert_planes(E, N, K, 300)
+    x = workloads.activations(T, K, 400, device=DEV)
+    tor, eor = workloads.top2_routing(T, E, 500)
+    y = dps.dps_moe_linear(mode, encs, x, torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV), p,
+                           r if mode else None)
+    ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r), threads=8)
+    assert rc == oracle.OK
+    assert_close_to_oracle(y, ref, f"moe E={E}")
+    assert dps.dps_stream_status() == dps.DPS_OK
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_identity_token_map_and_empty_experts(mode):
+    """token_of_row = NULL means row a reads x[a]; experts that receive no row are never touched."""
+    E, N, K, A = 6, 128, 256, 40
+    p, r, encs = expert_planes(E, N, K, 600)
+    x = workloads.activations(A, K, 700, device=DEV)
+    eor = np.random.default_rng(1).choice([0, 2, 5], A).astype(np.int32)     # experts 1, 3, 4 stay empty
+    y = dps.dps_moe_linear(mode, encs, x, None, torch.from_numpy(eor).to(DEV), p, r if mode else None)
+    ref, _ = oracle.moe_linear(mode, encs, to_np_words(x), None, eor, to_np_bytes(p), to_np_bytes(r), threads=8)
+    assert_close_to_oracle(y, ref, "identity map")
+
+
+def test_all_rows_one_expert_equals_dense():
+    E, N, K, A = 3, 256, 512, 70
+    p, r, encs = expert_planes(E, N, K, 800, mixed=False)
+    x = workloads.activations(A, K, 900, device=DEV)
+    eor = torch.full((A,), 1, dtype=torch.int32, device=DEV)
+    for mode in MODES:
+        y = dps.dps_moe_linear(mode, encs, x, None, eor, p, r if mode else None)
+        ref = oracle.linear(mode, encs[1], to_np_words(x), to_np_bytes(p[1]), to_np_bytes(r[1]), threads=8)
+        assert_close_to_oracle(y, ref, "one expert")
+
+
+def test_bad_indices_are_skipped_and_flagged():
+    E, N, K, T = 4, 64, 128, 8
+    p, r, encs = expert_planes(E, N, K, 1000)
+    x = workloads.activations(T, K, 1100, device=DEV)
+    tor, eor = workloads.top2_routing(T, E, 1200)
+    tor, eor = tor.copy(), eor.copy()
+    eor[3] = E
+    eor[6] = -1
+    tor[9] = T
+    y = torch.full((2 * T, N), 5.0, dtype=torch.float16, device=DEV)
+    dps.dps_moe_linear(dps.DPS_MODE_FULL, encs, x, torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV), p, r, y)
+    assert dps.dps_stream_status() == dps.binding.DPS_ERR_DATA
+    assert dps.dps_stream_status() == dps.DPS_OK                      # reading clears the word
+    ref, rc = oracle.moe_linear(dps.DPS_MODE_FULL, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r),
+                                y_init=np.full((2 * T, N), 5.0))
+    assert rc == oracle.ERR_DATA
+    got = y_as_f64(y)
+    for a in (3, 6, 9):
+        assert np.all(got[a] == 5.0)                                  # skipped rows are left untouched
+    assert_close_to_oracle(y, ref, "bad rows")
+
+
+def test_fast_mode_ignores_residual_and_is_deterministic():
+    E, N, K, T = 4, 128, 256, 24
+    p, r, encs = expert_planes(E, N, K, 1300)
+    x = workloads.activations(T, K, 1400, device=DEV)
+    tor, eor = workloads.top2_routing(T, E, 1500)
+    tor_d, eor_d = torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV)
+    a = dps.dps_moe_linear(dps.DPS_MODE_FAST, encs, x, tor_d, eor_d, p, None)
+    b = dps.dps_moe_linear(dps.DPS_MODE_FAST, encs, x, tor_d, eor_d, p, torch.full_like(r, 0xFF))
+    c = dps.dps_moe_linear(dps.DPS_MODE_FAST, encs, x, tor_d, eor_d, p, None)
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    assert torch.equal(a.view(torch.int16), c.view(torch.int16))
+
+
+def test_mixtral_shapes_sampled():
+    """Config 4 at full size: 8 experts, hidden 4096, ffn 14336, 256 tokens routed top-2.  The
+    oracle recomputes sampled entries of a few rows per expert."""
+    E, T = workloads.MIXTRAL_EXPERTS, workloads.MIXTRAL_TOKENS
+    tor, eor = workloads.top2_routing(T, E, 4200)
+    rng = np.random.default_rng(4999)
+    for li, (name, (N, K)) in enumerate(workloads.MIXTRAL_EXPERT.items()):
+        p = torch.empty((E, N, K), dtype=torch.uint8, device=DEV)
+        r = torch.empty((E, N, K), dtype=torch.uint8, device=DEV)
+        encs = []
+        for e in range(E):
+            w = workloads.weights(N, K, 4001 + 10 * li + e, device=DEV)
+            _, _, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO, p[e], r[e])
+            encs.append(enc)
+            del w
+        if name == "gate_up":
+            x = workloads.activations(T, K, 4100, device=DEV)
+            tmap = tor
+        else:
+            x = workloads.activations(2 * T, K, 4300, device=DEV)
+            tmap = None
+        tor_d = None if tmap is None else torch.from_numpy(tmap).to(DEV)
+        eor_d = torch.from_numpy(eor).to(DEV)
+        xn = to_np_words(x)
+        # rows to check: two rows of every expert
+        rows = np.concatenate([np.nonzero(eor == e)[0][:2] for e in range(E)])
+        cols = rng.integers(0, N, 48)
+        cols[:2] = [0, N - 1]
+        for mode in MODES:
+            y = dps.dps_moe_linear(mode, encs, x, tor_d, eor_d, p, r if mode else None)
+            got = y_as_f64(y)
+            for a in rows:
+                e = int(eor[a])
+                t = int(tmap[a]) if tmap is not None else int(a)
+                pe, re_ = to_np_bytes(p[e][cols.tolist()]), to_np_bytes(r[e][cols.tolist()])
+                ref = oracle.linear(mode, encs[e], xn[t:t + 1], pe, re_)[0]
+                scale = np.max(np.abs(ref))
+                assert np.max(np.abs(got[a, cols] - ref)) <= 2e-3 * scale, (name, mode, a)
+        assert dps.dps_stream_status() == dps.DPS_OK
+        del p, r
