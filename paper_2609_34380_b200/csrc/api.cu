@@ -1,6 +1,8 @@
 // The C ABI of libdps: argument validation, the per-device status word, and dispatch of each
 // call to a kernel family.  Nothing here allocates or frees device memory.
 #include <atomic>
+#include <cstdlib>
+#include <cstring>
 #include <mutex>
 
 #include "dps_internal.h"
@@ -40,6 +42,18 @@ DeviceInfo* device_info() {
         if (d.err == cudaSuccess) d.err = cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev);
     });
     return &d;
+}
+
+// Tuning / debugging knob: DPS_FORCE_PATH=gemv or =umma pins the dense kernel family.
+int forced_path() {
+    static const int path = [] {
+        const char* v = getenv("DPS_FORCE_PATH");
+        if (!v) return 0;
+        if (!strcmp(v, "gemv")) return 1;
+        if (!strcmp(v, "umma")) return 2;
+        return 0;
+    }();
+    return path;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -141,8 +155,13 @@ dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w
     if (st != DPS_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const uint8_t* r = (mode == DPS_MODE_FULL) ? w_resid : nullptr;  // fast mode never sees the pointer
-    if (launch_gemv(mode, enc, x, w_persist, r, y, M, N, K, stream) != cudaSuccess) return DPS_ERR_CUDA;
-    return DPS_OK;
+    // Up to four tokens the CUDA-core GEMV wins (no tensor-memory set-up, exact FP32 FMAs keep up
+    // with the weight stream); beyond that the tensor cores take the arithmetic.
+    const int path = forced_path();
+    const bool use_gemv = path == 1 || (path == 0 && M <= 4);
+    cudaError_t err = use_gemv ? launch_gemv(mode, enc, x, w_persist, r, y, M, N, K, stream)
+                               : launch_umma_linear(mode, enc, x, w_persist, r, y, M, N, K, d->status, stream);
+    return err == cudaSuccess ? DPS_OK : DPS_ERR_CUDA;
 }
 
 size_t dps_moe_workspace_bytes(int64_t A, int32_t E) { return moe_workspace_bytes(A, E); }

@@ -21,6 +21,11 @@ cudaError_t launch_reconstruct(const uint8_t* p, const uint8_t* r, uint16_t* w, 
 cudaError_t launch_gemv(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
                         int64_t M, int64_t N, int64_t K, cudaStream_t stream);
 
+// Dense linear, tensor-core path (tcgen05 + TMEM).  `status` receives DPS_ERR_CUDA if a bounded
+// wait inside the kernel ever gives up.
+cudaError_t launch_umma_linear(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
+                               int64_t M, int64_t N, int64_t K, int* status, cudaStream_t stream);
+
 // Grouped linear.
 size_t moe_workspace_bytes(int64_t A, int32_t E);
 cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const int32_t* token_of_row,
