@@ -5,17 +5,17 @@
 // residual tensor into the original FP16 values *during computation*; fast mode uses the FP8
 // tensor alone.  Here that combination happens on the way from shared memory to tensor memory.
 //
-// Tile: 128 weight rows (UMMA M) x TN tokens (UMMA N), K walked in blocks of 64.  The problem
+// Tile: 128 weight rows (UMMA M) x TN tokens (UMMA N), K walked in blocks of 128.  The problem
 // is "swapped": D[row][token] = sum_k W[row][k] * x[token][k], so that even a handful of decode
 // tokens fills the 128-lane datapath with weight rows and every weight byte is fetched once.
 //
 // Roles (6 warps):
-//   warp 0     TMA producer: P tile (128 x 64 bytes), R tile (full mode), x tile (TN x 64 halves)
+//   warp 0     TMA producer: P tile (128 x 128 bytes), R tile (full mode), x tile (TN x 128 halves)
 //              into a ring of shared-memory stages, completion counted on mbarriers.
 //   warp 1     allocates tensor memory; one lane issues tcgen05.mma (A from TMEM, B from smem)
 //              and commits stage-release barriers.
 //   warps 2-5  "zip" warps: each owns 32 TMEM lanes = 32 weight rows.  Per K block a thread
-//              reads its row's 64 plane bytes (swizzled, conflict-free), rebuilds 64 FP16 words
+//              reads its row's 128 plane bytes (swizzled, conflict-free), rebuilds 128 FP16 words
 //              in registers with byte permutes and writes them to the A ring in TMEM with one
 //              tcgen05.st.  After the K loop the same warps drain the accumulator
 //              (tcgen05.ld), round to FP16 and store y.
@@ -23,6 +23,7 @@
 // instead of 5-6, and the tensor core reads only the small activation tile from it.
 #include <cuda_fp16.h>
 
+#include <cstdio>
 #include <cstdlib>
 
 #include "bits.cuh"
@@ -36,11 +37,13 @@ namespace {
 using namespace sm100;
 
 constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
-constexpr int kBlockK = 64;      // K elements per pipeline stage
-constexpr int kAStages = 4;      // A ring in tensor memory (32 columns each)
+constexpr int kBlockK = 128;     // K elements per pipeline stage: 128-byte plane rows, the widest swizzled TMA box
+constexpr int kXAtoms = kBlockK / 64;  // the x tile is stored as 64-element (128-byte) swizzle atoms
+constexpr int kACols = kBlockK / 2;    // TMEM columns of one A stage (two FP16 per column)
+constexpr int kAStages = 2;      // A ring in tensor memory
 constexpr int kZipGroups = 2;    // groups of 4 zip warps; group g takes K blocks g, g + G, ...
 constexpr int kThreads = 64 + kZipGroups * 128;
-constexpr int kPlaneStageBytes = kTileRows * kBlockK;  // 8 KB per plane per stage
+constexpr int kPlaneStageBytes = kTileRows * kBlockK;  // 16 KB per plane per stage
 constexpr int kMaxStages = 12;
 constexpr int kMaxSplit = 8;     // portable cluster size
 static_assert(kAStages % kZipGroups == 0, "each A stage must belong to one zip group");
@@ -49,11 +52,33 @@ __host__ __device__ constexpr int stage_bytes(bool full, int tn) {
     return kPlaneStageBytes * (full ? 2 : 1) + tn * kBlockK * 2;
 }
 __host__ __device__ constexpr int tmem_cols(int tn) {
-    int need = tn + kAStages * 32;
+    int need = tn + kAStages * kACols;
     int c = 32;
     while (c < need) c <<= 1;
     return c;
 }
+
+// Optional timeline trace (compile with -DDPS_TRACE): lane 0 of each role of CTA (0,0,0) stamps
+// the SM clock at pipeline events of every K block.  Read back with dps_debug_trace().
+#ifdef DPS_TRACE
+constexpr int kTraceBlocks = 64, kTraceEvents = 16;
+__device__ long long g_trace[kTraceBlocks * kTraceEvents];
+__device__ unsigned long long g_cta_times[2048 * 8];
+#define DPS_CTA_STAMP(ev)                                                                          \
+    do {                                                                                           \
+        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);           \
+        if (threadIdx.x == 64 && cta_ < 2048) g_cta_times[cta_ * 8 + (ev)] = global_timer_ns();    \
+    } while (0)
+#define DPS_STAMP(ev, i)                                                                          \
+    do {                                                                                          \
+        if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 31) == 0 &&   \
+            (i) < kTraceBlocks)                                                                   \
+            g_trace[(i) * kTraceEvents + (ev)] = clock64();                                       \
+    } while (0)
+#else
+#define DPS_STAMP(ev, i) do { } while (0)
+#define DPS_CTA_STAMP(ev) do { } while (0)
+#endif
 
 struct UmmaParams {
     __half* y;
@@ -61,10 +86,11 @@ struct UmmaParams {
     int num_stages;
     int split;       // K split = cluster size along z; partial tiles are summed through DSMEM
     int* status;
+
 };
 
 template <int ENC, bool FULL, int TN>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, (tmem_cols(TN) <= 256 ? 2 : 1))
 umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
                    const __grid_constant__ CUtensorMap map_x, const UmmaParams prm) {
     constexpr int kStage = stage_bytes(FULL, TN);
@@ -80,6 +106,15 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     __shared__ __align__(8) uint64_t bar_d_full;
     __shared__ uint32_t tmem_base_slot;
 
+    DPS_CTA_STAMP(0);
+#ifdef DPS_TRACE
+    {
+        unsigned smid_;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_));
+        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+        if (threadIdx.x == 64 && cta_ < 2048) g_cta_times[cta_ * 8 + 5] = smid_;
+    }
+#endif
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_stages = prm.num_stages;
@@ -88,9 +123,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const int total_kb = (prm.K + kBlockK - 1) / kBlockK;
     const int split = prm.split;
     const int rank = (split > 1) ? (int)cluster_ctarank() : 0;   // == blockIdx.z
-    const int kb_begin = (int)((int64_t)total_kb * rank / split);
-    const int kb_end = (int)((int64_t)total_kb * (rank + 1) / split);
-    const int num_kb = kb_end - kb_begin;
+    // K blocks are dealt round-robin to the CTAs of the cluster: at any moment the cluster reads
+    // `split` adjacent 64-byte pieces of each weight row, which DRAM serves as one longer burst.
+    const int num_kb = (total_kb - rank + split - 1) / split;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < num_stages; ++s) {
@@ -111,9 +146,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    DPS_CTA_STAMP(1);
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_d = tmem_base;           // TN accumulator columns
-    const uint32_t tmem_a = tmem_base + TN;      // kAStages x 32 columns of packed FP16 pairs
+    const uint32_t tmem_a = tmem_base + TN;      // kAStages x kACols columns of packed FP16 pairs
 
     // Partial tile for the split-K sum, token-major: red[token][row].  It overlays the stage ring,
     // which is idle once the accumulator is complete.
@@ -121,40 +157,62 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
 
     bool ok = true;
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
-        if (lane == 0) {
-            for (int i = 0; i < num_kb && ok; ++i) {
-                const int s = i % num_stages;
-                const uint32_t ph = (uint32_t)(i / num_stages) & 1u;
+        // ---------------- TMA producer (whole warp converged, one elected lane issues) ----------------
+        // Stages are filled two at a time when the ring is deep enough: the two boxes cover 256
+        // adjacent bytes of every weight row, which DRAM serves noticeably better than 128.
+        const bool pair = (num_stages >= 4) && (num_stages % 2 == 0);
+        for (int i = 0; i < num_kb && ok; ++i) {
+            const int s = i % num_stages;
+            const uint32_t ph = (uint32_t)(i / num_stages) & 1u;
+            if (!pair || (i & 1) == 0) {
                 ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);
-                if (!ok) break;
+                if (ok && pair && i + 1 < num_kb)
+                    ok = mbar_wait(smem_u32(&bar_empty[(i + 1) % num_stages]),
+                                   ((uint32_t)((i + 1) / num_stages) & 1u) ^ 1u);
+            }
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            DPS_STAMP(0, i);
+            if (elect_one()) {
                 const uint32_t full = smem_u32(&bar_full[s]);
                 const uint32_t dst = smem_base + (uint32_t)s * kStage;
-                const int k = (kb_begin + i) * kBlockK;
+                const int k = (rank + i * split) * kBlockK;
                 mbar_arrive_expect_tx(full, (uint32_t)kStage);
                 tma_load_2d(dst, &map_p, full, k, n0);
                 if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, n0);
-                tma_load_2d(dst + kXOffset, &map_x, full, k, m0);
+#pragma unroll
+                for (int t = 0; t < kXAtoms; ++t)
+                    tma_load_2d(dst + kXOffset + (uint32_t)(t * TN * 128), &map_x, full, k + t * 64, m0);
             }
+            __syncwarp();
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            for (int i = 0; i < num_kb && ok; ++i) {
-                const int s = i % num_stages, a = i % kAStages;
-                ok = mbar_wait(smem_u32(&bar_full[s]), (uint32_t)(i / num_stages) & 1u);
-                if (ok) ok = mbar_wait(smem_u32(&bar_a_full[a]), (uint32_t)(i / kAStages) & 1u);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint64_t bdesc = umma_desc_k_sw128(smem_base + (uint32_t)s * kStage + kXOffset);
+        // ---------------- MMA issuer (whole warp converged, one elected lane issues) ----------------
+        for (int i = 0; i < num_kb && ok; ++i) {
+            const int s = i % num_stages, a = i % kAStages;
+            ok = mbar_wait(smem_u32(&bar_full[s]), (uint32_t)(i / num_stages) & 1u);
+            DPS_STAMP(1, i);
+            if (ok) ok = mbar_wait(smem_u32(&bar_a_full[a]), (uint32_t)(i / kAStages) & 1u);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            DPS_STAMP(2, i);
+            tc_fence_after_sync();
+            if (elect_one()) {
+                const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
 #pragma unroll
-                for (int j = 0; j < kBlockK / 16; ++j)
-                    umma_f16_ts(tmem_d, tmem_a + (uint32_t)(a * 32 + j * 8), bdesc + (uint64_t)(j * 2), kIdesc,
+                for (int j = 0; j < kBlockK / 16; ++j) {
+                    // 16 K elements = 32 bytes inside the 128-byte swizzle atom (j / 4)
+                    const uint64_t bdesc = umma_desc_k_sw128(xbase + (uint32_t)((j >> 2) * TN * 128)) +
+                                           (uint64_t)((j & 3) * 2);
+                    umma_f16_ts(tmem_d, tmem_a + (uint32_t)(a * kACols + j * 8), bdesc, kIdesc,
                                 (i > 0 || j > 0) ? 1u : 0u);
+                }
                 umma_commit(smem_u32(&bar_empty[s]));
                 umma_commit(smem_u32(&bar_a_empty[a]));
+                if (i == num_kb - 1) umma_commit(smem_u32(&bar_d_full));
             }
-            if (ok) umma_commit(smem_u32(&bar_d_full));
+            __syncwarp();
+            DPS_STAMP(3, i);
         }
     } else {
         // ---------------- zip warps: planes -> FP16 -> tensor memory; then epilogue ----------------
@@ -162,18 +220,21 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         const int q = warp & 3;                  // TMEM lane quarter this warp may touch
         const int row = q * 32 + lane;           // weight row inside the tile
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-        const uint32_t sw = (uint32_t)((row >> 1) & 3);  // 64-byte swizzle: chunk ^= (row / 2) % 4
+        const uint32_t sw = (uint32_t)(row & 7);  // 128-byte swizzle: 16-byte chunk index ^= row % 8
         for (int i = group; i < num_kb && ok; i += kZipGroups) {
             const int s = i % num_stages, a = i % kAStages;
+            if (warp == 2 + 4 * group) DPS_STAMP(4, i);
             ok = mbar_wait(smem_u32(&bar_full[s]), (uint32_t)(i / num_stages) & 1u);
+            if (warp == 2 + 4 * group) DPS_STAMP(5, i);
             if (ok) ok = mbar_wait(smem_u32(&bar_a_empty[a]), ((uint32_t)(i / kAStages) & 1u) ^ 1u);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
+            if (warp == 2 + 4 * group) DPS_STAMP(6, i);
             tc_fence_after_sync();
             const uint32_t prow = smem_base + (uint32_t)s * kStage + (uint32_t)row * kBlockK;
-            uint32_t h[32];
+            uint32_t h[kACols];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < kBlockK / 16; ++c) {
                 const uint32_t off = ((uint32_t)c ^ sw) * 16u;
                 uint4 pv, rv = make_uint4(0, 0, 0, 0);
                 asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -188,7 +249,14 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
 #pragma unroll
                 for (int j = 0; j < 8; ++j) h[c * 8 + j] = h8[j];
             }
-            tmem_st_32x32b_x32(tmem_a + lane_base + (uint32_t)(a * 32), h);
+#pragma unroll
+            for (int t = 0; t < kACols / 32; ++t) {
+                uint32_t part[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) part[j] = h[t * 32 + j];
+                tmem_st_32x32b_x32(tmem_a + lane_base + (uint32_t)(a * kACols + t * 32), part);
+            }
+            if (warp == 2 + 4 * group) DPS_STAMP(7, i);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
@@ -196,11 +264,13 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 mbar_arrive(smem_u32(&bar_a_full[a]));
                 mbar_arrive(smem_u32(&bar_empty[s]));
             }
+            if (warp == 2 + 4 * group) DPS_STAMP(8, i);
         }
         // epilogue (first zip group): D[row][token] -> y[token][n0 + row], or -> red for split K
         if (group == 0) {
             if (ok) ok = mbar_wait(smem_u32(&bar_d_full), 0u);
             ok = __all_sync(0xFFFFFFFFu, ok);
+            DPS_CTA_STAMP(2);
             if (ok) {
                 tc_fence_after_sync();
                 const int n = n0 + row;
@@ -224,6 +294,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         }
     }
     if (!ok) atomicExch(prm.status, (int)DPS_ERR_CUDA);
+    DPS_CTA_STAMP(3);
 
     if (split > 1) {
         // Split-K: every CTA of the cluster holds a partial tile in its shared memory.  CTA `rank`
@@ -231,6 +302,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         // result is deterministic) straight out of its peers' shared memory.
         __syncthreads();
         cluster_sync_all();
+        DPS_CTA_STAMP(4);
         const uint32_t red_addr = smem_base;
         for (int e = threadIdx.x; e < (TN / 1) * kTileRows; e += kThreads) {
             const int c = e / kTileRows, r = e % kTileRows;
@@ -244,12 +316,14 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         }
         cluster_sync_all();
     }
+    DPS_CTA_STAMP(6);
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kCols);
     }
+    DPS_CTA_STAMP(7);
 }
 
 // ---- host side ---------------------------------------------------------------------------------
@@ -293,13 +367,13 @@ bool make_map_2d(CUtensorMap* map, const void* base, CUtensorMapDataType dt, int
 }
 
 // K split for a launch of `tiles` output tiles: the factor (<= 8, a portable cluster) that fills
-// the machine's CTA slots most evenly, keeping at least 6 K blocks per CTA; ties go to the
+// the machine's CTA slots most evenly, keeping at least 4 K blocks per CTA; ties go to the
 // smaller factor (less reduction traffic).
 int choose_split(int64_t tiles, int total_kb, int slots) {
     int best = 1;
     double best_eff = 0.0;
     for (int s = 1; s <= kMaxSplit; ++s) {
-        if (s > 1 && total_kb / s < 6) break;
+        if (s > 1 && total_kb / s < 4) break;
         const int64_t units = tiles * s;
         const int64_t waves = (units + slots - 1) / slots;
         const double eff = (double)units / (double)(waves * slots);
@@ -316,30 +390,37 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
                       int* status, cudaStream_t stream) {
     constexpr int kStage = stage_bytes(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(TN) <= 256 ? 2 : 1;
-    constexpr int kSmemBudget = kCtasPerSm == 2 ? 100 * 1024 : 200 * 1024;
+    constexpr int kSmemBudget = kCtasPerSm == 2 ? 110 * 1024 : 216 * 1024;
     int stages = kSmemBudget / kStage;
     if (stages > 8) stages = 8;
-    if (stages < 3) stages = 3;
+    if (stages < 2) stages = 2;
+    stages -= stages % kZipGroups;  // a stage always belongs to the same zip group, so that every
+                                    // waiter sees every phase of the barriers it waits on
     const size_t smem = (size_t)stages * kStage + 1024;
     static bool configured = false;  // per instantiation
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(umma_linear_kernel<ENC, FULL, TN>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        if (e != cudaSuccess) return e;
+        // Ask for the largest shared-memory carve-out, otherwise the driver sizes it for ONE CTA of
+        // this kernel and a second CTA never becomes resident on the SM.
+        e = cudaFuncSetAttribute(umma_linear_kernel<ENC, FULL, TN>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;
     }
     CUtensorMap mp, mr, mx;
     if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, (uint64_t)K, kTileRows, kBlockK,
-                     CU_TENSOR_MAP_SWIZZLE_64B))
+                     CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
     if (FULL) {
         if (!make_map_2d(&mr, r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, (uint64_t)K, kTileRows, kBlockK,
-                         CU_TENSOR_MAP_SWIZZLE_64B))
+                         CU_TENSOR_MAP_SWIZZLE_128B))
             return cudaErrorInvalidValue;
     } else {
         mr = mp;
     }
-    if (!make_map_2d(&mx, x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)M, (uint64_t)K, TN, kBlockK,
+    if (!make_map_2d(&mx, x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)M, (uint64_t)K, TN, 64,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
     const int64_t row_tiles = (N + kTileRows - 1) / kTileRows, tok_tiles = (M + TN - 1) / TN;
@@ -358,6 +439,20 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     prm.split = split;
     prm.status = status;
 
+#ifdef DPS_TRACE
+    {
+        static bool printed = false;
+        if (!printed) {
+            printed = true;
+            cudaFuncAttributes fa;
+            cudaFuncGetAttributes(&fa, umma_linear_kernel<ENC, FULL, TN>);
+            int nb = -1;
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, umma_linear_kernel<ENC, FULL, TN>, kThreads, smem);
+            fprintf(stderr, "[trace] TN=%d regs=%d static_smem=%zu dyn=%zu maxdyn=%d carveout=%d occupancy=%d stages=%d\n", TN,
+                    fa.numRegs, fa.sharedSizeBytes, smem, fa.maxDynamicSharedSizeBytes, fa.preferredShmemCarveout, nb, stages);
+        }
+    }
+#endif
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     cfg.blockDim = dim3(kThreads, 1, 1);
@@ -386,6 +481,16 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
 }
 
 }  // namespace
+
+#ifdef DPS_TRACE
+extern "C" __attribute__((visibility("default"))) int dps_debug_trace(long long* out, int max_words) {
+    const int n = max_words < kTraceBlocks * kTraceEvents ? max_words : kTraceBlocks * kTraceEvents;
+    return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * n);
+}
+extern "C" __attribute__((visibility("default"))) int dps_debug_cta_times(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_cta_times, sizeof(unsigned long long) * 2048 * 8);
+}
+#endif
 
 cudaError_t launch_umma_linear(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
                                int64_t M, int64_t N, int64_t K, int* status, cudaStream_t stream) {
