@@ -69,12 +69,16 @@ __device__ unsigned long long g_cta_times[2048 * 8];
         const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);           \
         if (threadIdx.x == 64 && cta_ < 2048) g_cta_times[cta_ * 8 + (ev)] = global_timer_ns();    \
     } while (0)
+#ifdef DPS_TRACE_BLOCKS
 #define DPS_STAMP(ev, i)                                                                          \
     do {                                                                                          \
         if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (threadIdx.x & 31) == 0 &&   \
             (i) < kTraceBlocks)                                                                   \
             g_trace[(i) * kTraceEvents + (ev)] = clock64();                                       \
     } while (0)
+#else
+#define DPS_STAMP(ev, i) do { } while (0)
+#endif
 #else
 #define DPS_STAMP(ev, i) do { } while (0)
 #define DPS_CTA_STAMP(ev) do { } while (0)
@@ -85,6 +89,7 @@ struct UmmaParams {
     int M, N, K;
     int num_stages;
     int split;       // K split = cluster size along z; partial tiles are summed through DSMEM
+    int red_offset;  // byte offset (from the aligned base of dynamic smem) of the split-K mailbox
     int* status;
 
 };
@@ -106,6 +111,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     __shared__ __align__(8) uint64_t bar_d_full;
     __shared__ uint32_t tmem_base_slot;
 
+    grid_launch_dependents();  // the next kernel's prologue may overlap this kernel's tail
     DPS_CTA_STAMP(0);
 #ifdef DPS_TRACE
     {
@@ -151,16 +157,23 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const uint32_t tmem_d = tmem_base;           // TN accumulator columns
     const uint32_t tmem_a = tmem_base + TN;      // kAStages x kACols columns of packed FP16 pairs
 
-    // Partial tile for the split-K sum, token-major: red[token][row].  It overlays the stage ring,
-    // which is idle once the accumulator is complete.
+    // Split-K sums.  TN <= 64 ("push"): every CTA owns the tokens c with c % split == rank and has a
+    // mailbox mail[source rank][slot = c / split][row] in its own shared memory, outside the stage
+    // ring; peers store their partial sums straight into it, one cluster barrier later the owner
+    // adds them in rank order.  TN >= 128 ("pull"): the partial tile red[token][row] overlays the
+    // idle stage ring and owners read it out of their peers' memory between two cluster barriers.
+    constexpr bool kPush = TN <= 64;
     float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
+    const uint32_t mail_addr = smem_base + (uint32_t)prm.red_offset;
+    const int slots = (TN + split - 1) / split;
 
     bool ok = true;
     if (warp == 0) {
         // ---------------- TMA producer (whole warp converged, one elected lane issues) ----------------
         // Stages are filled two at a time when the ring is deep enough: the two boxes cover 256
         // adjacent bytes of every weight row, which DRAM serves noticeably better than 128.
-        const bool pair = (num_stages >= 4) && (num_stages % 2 == 0);
+        const bool pair = (num_stages >= 6) && (num_stages % 2 == 0);
+        grid_dependency_wait();  // everything read from global memory may come from the preceding kernel
         for (int i = 0; i < num_kb && ok; ++i) {
             const int s = i % num_stages;
             const uint32_t ph = (uint32_t)(i / num_stages) & 1u;
@@ -279,7 +292,14 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                     uint32_t v[16];
                     tmem_ld_32x32b_x16(tmem_d + lane_base + (uint32_t)c0, v);
                     tmem_wait_ld();
-                    if (split > 1) {
+                    if (split > 1 && kPush) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int c = c0 + j, owner = c % split, slot = c / split;
+                            const uint32_t local = mail_addr + (uint32_t)(((rank * slots + slot) * kTileRows + row) * 4);
+                            st_cluster_f32(map_to_cta(local, (uint32_t)owner), __uint_as_float(v[j]));
+                        }
+                    } else if (split > 1) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j) red[(c0 + j) * kTileRows + row] = __uint_as_float(v[j]);
                     } else if (n < prm.N) {
@@ -296,15 +316,26 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     if (!ok) atomicExch(prm.status, (int)DPS_ERR_CUDA);
     DPS_CTA_STAMP(3);
 
-    if (split > 1) {
-        // Split-K: every CTA of the cluster holds a partial tile in its shared memory.  CTA `rank`
-        // sums tokens rank, rank + split, ... over all partials in rank order (fixed order, so the
-        // result is deterministic) straight out of its peers' shared memory.
+    if (split > 1 && kPush) {
+        __syncthreads();
+        cluster_sync_all();  // release/acquire: every peer's stores into this CTA's mailbox are visible
+        DPS_CTA_STAMP(4);
+        const float* mail = reinterpret_cast<const float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + prm.red_offset);
+        for (int e = threadIdx.x; e < slots * kTileRows; e += kThreads) {
+            const int slot = e / kTileRows, r = e % kTileRows;
+            const int c = slot * split + rank;
+            const int m = m0 + c, n = n0 + r;
+            if (c >= TN || m >= prm.M || n >= prm.N) continue;
+            float acc = 0.f;
+            for (int j = 0; j < split; ++j) acc += mail[(j * slots + slot) * kTileRows + r];
+            prm.y[(int64_t)m * prm.N + n] = __float2half_rn(acc);
+        }
+    } else if (split > 1) {
         __syncthreads();
         cluster_sync_all();
         DPS_CTA_STAMP(4);
         const uint32_t red_addr = smem_base;
-        for (int e = threadIdx.x; e < (TN / 1) * kTileRows; e += kThreads) {
+        for (int e = threadIdx.x; e < TN * kTileRows; e += kThreads) {
             const int c = e / kTileRows, r = e % kTileRows;
             if ((c % split) != rank) continue;
             const int m = m0 + c, n = n0 + r;
@@ -314,7 +345,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 acc += ld_cluster_f32(map_to_cta(red_addr + (uint32_t)(c * kTileRows + r) * 4u, (uint32_t)j));
             prm.y[(int64_t)m * prm.N + n] = __float2half_rn(acc);
         }
-        cluster_sync_all();
+        cluster_sync_all();  // nobody leaves while a peer may still read its partial tile
     }
     DPS_CTA_STAMP(6);
     tc_fence_before_sync();
@@ -366,21 +397,16 @@ bool make_map_2d(CUtensorMap* map, const void* base, CUtensorMapDataType dt, int
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// K split for a launch of `tiles` output tiles: the factor (<= 8, a portable cluster) that fills
-// the machine's CTA slots most evenly, keeping at least 4 K blocks per CTA; ties go to the
-// smaller factor (less reduction traffic).
-int choose_split(int64_t tiles, int total_kb, int slots) {
+// K split for a launch of `tiles` output tiles.  capacity[s] = CTAs that can be resident at once
+// when launched as clusters of s (clusters must fit inside one GPC, so this is not a multiple of
+// the SM count).  Measured on B200: a second wave costs more than it buys, so take the largest
+// factor (<= 8, a portable cluster) whose CTAs are all resident at once, keeping at least 4 K
+// blocks per CTA.
+int choose_split(int64_t tiles, int total_kb, const int* capacity) {
     int best = 1;
-    double best_eff = 0.0;
-    for (int s = 1; s <= kMaxSplit; ++s) {
-        if (s > 1 && total_kb / s < 4) break;
-        const int64_t units = tiles * s;
-        const int64_t waves = (units + slots - 1) / slots;
-        const double eff = (double)units / (double)(waves * slots);
-        if (eff > best_eff + 0.02) {
-            best_eff = eff;
-            best = s;
-        }
+    for (int s = 2; s <= kMaxSplit; ++s) {
+        if (total_kb / s < 4) break;
+        if (tiles * s <= capacity[s]) best = s;
     }
     return best;
 }
@@ -390,23 +416,49 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
                       int* status, cudaStream_t stream) {
     constexpr int kStage = stage_bytes(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(TN) <= 256 ? 2 : 1;
-    constexpr int kSmemBudget = kCtasPerSm == 2 ? 110 * 1024 : 216 * 1024;
-    int stages = kSmemBudget / kStage;
+    constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
+    constexpr int kMailBytes = TN <= 64 ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox
+    int stages = (kSmemTotal - kMailBytes) / kStage;
     if (stages > 8) stages = 8;
     if (stages < 2) stages = 2;
     stages -= stages % kZipGroups;  // a stage always belongs to the same zip group, so that every
                                     // waiter sees every phase of the barriers it waits on
-    const size_t smem = (size_t)stages * kStage + 1024;
-    static bool configured = false;  // per instantiation
+    const size_t smem = (size_t)stages * kStage + kMailBytes + 1024;
+    auto kernel = umma_linear_kernel<ENC, FULL, TN>;
+    static int capacity[kMaxSplit + 1] = {0};  // per instantiation; filled on first use
+    static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(umma_linear_kernel<ENC, FULL, TN>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
         if (e != cudaSuccess) return e;
-        // Ask for the largest shared-memory carve-out, otherwise the driver sizes it for ONE CTA of
-        // this kernel and a second CTA never becomes resident on the SM.
-        e = cudaFuncSetAttribute(umma_linear_kernel<ENC, FULL, TN>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        // Ask for the largest shared-memory carve-out, otherwise the driver may size it for ONE CTA
+        // of this kernel and a second CTA never becomes resident on the SM.
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
+        for (int s = 1; s <= kMaxSplit; ++s) {
+            cudaLaunchConfig_t q = {};
+            q.gridDim = dim3(1, 1, (unsigned)s);
+            q.blockDim = dim3(kThreads, 1, 1);
+            q.dynamicSmemBytes = smem;
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = 1;
+            qa[0].val.clusterDim.y = 1;
+            qa[0].val.clusterDim.z = (unsigned)s;
+            q.attrs = qa;
+            q.numAttrs = 1;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &q) != cudaSuccess) clusters = 0;
+            capacity[s] = clusters * s;
+        }
+        (void)cudaGetLastError();
+        // The query can be more conservative about CTAs per SM than the hardware turns out to be
+        // (it reported one where two were measured resident); keep its GPC packing ratios and
+        // rescale to the CTAs per SM this kernel is sized for.
+        const int slots = sm_count() * kCtasPerSm;
+        if (capacity[1] <= 0) capacity[1] = slots;
+        const int base = capacity[1];
+        for (int s = 1; s <= kMaxSplit; ++s) capacity[s] = (int)((int64_t)capacity[s] * slots / base);
         configured = true;
     }
     CUtensorMap mp, mr, mx;
@@ -426,10 +478,14 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     const int64_t row_tiles = (N + kTileRows - 1) / kTileRows, tok_tiles = (M + TN - 1) / TN;
     const int total_kb = (int)((K + kBlockK - 1) / kBlockK);
     int split = forced_split();
-    if (split <= 0) split = choose_split(row_tiles * tok_tiles, total_kb, sm_count() * kCtasPerSm);
+    if (split <= 0) split = choose_split(row_tiles * tok_tiles, total_kb, capacity);
     if (split > total_kb) split = total_kb;
     if (split > kMaxSplit) split = kMaxSplit;
-    if ((size_t)stages * kStage < (size_t)TN * kTileRows * 4) split = 1;  // partial tile overlays the stage ring
+    if (kMailBytes == 0 && (size_t)stages * kStage < (size_t)TN * kTileRows * 4) split = 1;  // pull mode overlays the ring
+    if (getenv("DPS_DEBUG"))
+        fprintf(stderr, "[dps] umma TN=%d full=%d N=%lld K=%lld M=%lld stages=%d split=%d capacity=%d,%d,%d,%d,%d,%d,%d,%d\n",
+                TN, (int)FULL, (long long)N, (long long)K, (long long)M, stages, split, capacity[1], capacity[2],
+                capacity[3], capacity[4], capacity[5], capacity[6], capacity[7], capacity[8]);
     UmmaParams prm;
     prm.y = static_cast<__half*>(y);
     prm.M = (int)M;
@@ -437,35 +493,26 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     prm.K = (int)K;
     prm.num_stages = stages;
     prm.split = split;
+    prm.red_offset = stages * kStage;
     prm.status = status;
 
-#ifdef DPS_TRACE
-    {
-        static bool printed = false;
-        if (!printed) {
-            printed = true;
-            cudaFuncAttributes fa;
-            cudaFuncGetAttributes(&fa, umma_linear_kernel<ENC, FULL, TN>);
-            int nb = -1;
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, umma_linear_kernel<ENC, FULL, TN>, kThreads, smem);
-            fprintf(stderr, "[trace] TN=%d regs=%d static_smem=%zu dyn=%zu maxdyn=%d carveout=%d occupancy=%d stages=%d\n", TN,
-                    fa.numRegs, fa.sharedSizeBytes, smem, fa.maxDynamicSharedSizeBytes, fa.preferredShmemCarveout, nb, stages);
-        }
-    }
-#endif
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = (unsigned)split;
+    // Programmatic dependent launch: this kernel may start while the previous one drains; it
+    // waits (griddepcontrol.wait) before its first global read.
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, umma_linear_kernel<ENC, FULL, TN>, mp, mr, mx, prm);
+    cfg.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, prm);
     count_launch();
     return e;
 }
