@@ -117,8 +117,9 @@ DPS_API dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const ui
  * x: [T][K] FP16.  y: [A][N] FP16.  w_persist / w_resid: [E][N][K] bytes (w_resid may be
  * NULL in FAST mode).  enc_per_expert: HOST array of E encodings (E4M3 or E5M2), read
  * before the call returns.  token_of_row (may be NULL) and expert_of_row: device int32[A].
- * workspace: device scratch of at least dps_moe_workspace_bytes(A, E) bytes, 16-byte
- * aligned, owned by the caller; its contents are overwritten.  A row whose expert is
+ * workspace: device scratch of at least dps_moe_workspace_bytes(A, E, K) bytes, 16-byte
+ * aligned, owned by the caller; its contents are overwritten (routing tables and the
+ * activations regrouped by expert).  E may not exceed 1024.  A row whose expert is
  * outside [0, E) or whose token is outside [0, T) is skipped and flagged (see
  * dps_stream_status).  A == 0 returns DPS_OK without a launch.  Never synchronises.
  */
@@ -128,8 +129,9 @@ DPS_API dps_status dps_moe_linear(int32_t mode, const int32_t* enc_per_expert, c
                           int64_t A, int64_t T, int64_t N, int64_t K, int32_t E,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Bytes of scratch dps_moe_linear needs for A rows and E experts (0 if A or E is invalid). */
-DPS_API size_t dps_moe_workspace_bytes(int64_t A, int32_t E);
+/* Bytes of scratch dps_moe_linear needs for A rows, E experts and K inputs (0 if an argument is
+ * invalid). */
+DPS_API size_t dps_moe_workspace_bytes(int64_t A, int32_t E, int64_t K);
 
 /*
  * Synchronises the stream, then returns and clears the current device's status word:

@@ -28,7 +28,7 @@ ABI = {
     "dps_linear": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "dps_moe_linear": (ctypes.c_int, [_i32, ctypes.POINTER(_i32), _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64,
                                       _i64, _i32, _vp, ctypes.c_size_t, _vp]),
-    "dps_moe_workspace_bytes": (ctypes.c_size_t, [_i64, _i32]),
+    "dps_moe_workspace_bytes": (ctypes.c_size_t, [_i64, _i32, _i64]),
     "dps_stream_status": (ctypes.c_int, [_vp]),
     "dps_launch_count": (_i64, []),
     "dps_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -133,8 +133,8 @@ def dps_linear(mode: int, enc: int, x: torch.Tensor, w_persist: torch.Tensor, w_
     return y
 
 
-def dps_moe_workspace_bytes(A: int, E: int) -> int:
-    return int(library().dps_moe_workspace_bytes(int(A), int(E)))
+def dps_moe_workspace_bytes(A: int, E: int, K: int) -> int:
+    return int(library().dps_moe_workspace_bytes(int(A), int(E), int(K)))
 
 
 def dps_moe_linear(mode: int, enc_per_expert: Sequence[int], x: torch.Tensor, token_of_row: Optional[torch.Tensor],
@@ -150,7 +150,7 @@ def dps_moe_linear(mode: int, enc_per_expert: Sequence[int], x: torch.Tensor, to
     if y is None:
         y = torch.empty((A, N), dtype=torch.float16, device=x.device)
     if workspace is None:
-        workspace = torch.empty(max(dps_moe_workspace_bytes(A, E), 16), dtype=torch.uint8, device=x.device)
+        workspace = torch.empty(max(dps_moe_workspace_bytes(A, E, K), 16), dtype=torch.uint8, device=x.device)
     enc_arr = (_i32 * E)(*[int(e) for e in enc_per_expert])
     st = library().dps_moe_linear(int(mode), enc_arr, _dev(x, torch.float16, "x"),
                                   _dev(token_of_row, torch.int32, "token_of_row"),

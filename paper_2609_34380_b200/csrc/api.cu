@@ -164,7 +164,7 @@ dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w
     return err == cudaSuccess ? DPS_OK : DPS_ERR_CUDA;
 }
 
-size_t dps_moe_workspace_bytes(int64_t A, int32_t E) { return moe_workspace_bytes(A, E); }
+size_t dps_moe_workspace_bytes(int64_t A, int32_t E, int64_t K) { return moe_workspace_bytes(A, E, K); }
 
 dps_status dps_moe_linear(int32_t mode, const int32_t* enc_per_expert, const void* x, const int32_t* token_of_row,
                           const int32_t* expert_of_row, const uint8_t* w_persist, const uint8_t* w_resid, void* y,
@@ -175,7 +175,7 @@ dps_status dps_moe_linear(int32_t mode, const int32_t* enc_per_expert, const voi
     if (A > ((int64_t)1 << 30) || T > ((int64_t)1 << 30) || N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31))
         return DPS_ERR_SHAPE;
     if (!enc_per_expert) return DPS_ERR_NULL;
-    const size_t need = moe_workspace_bytes(A, E);
+    const size_t need = moe_workspace_bytes(A, E, K);
     if (need == 0) return DPS_ERR_SHAPE;
     for (int32_t e = 0; e < E; ++e)
         if (enc_per_expert[e] != DPS_ENC_E4M3 && enc_per_expert[e] != DPS_ENC_E5M2) return DPS_ERR_ENCODING;

@@ -26,8 +26,17 @@ cudaError_t launch_gemv(int mode, int enc, const void* x, const uint8_t* p, cons
 cudaError_t launch_umma_linear(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
                                int64_t M, int64_t N, int64_t K, int* status, cudaStream_t stream);
 
+// Grouped linear on the tensor-core path.  x_sorted: [A][K] activations grouped by expert;
+// tiles / num_tiles / sorted_rows: device tables built by the routing pre-pass; tn: token-tile
+// width the tile list was built for (grouped_tile_tokens); max_tiles: upper bound on num_tiles.
+int grouped_tile_tokens(int64_t A, int32_t E);
+cudaError_t launch_umma_grouped(int mode, const uint32_t* e5m2_mask, const void* x_sorted, const uint8_t* p,
+                                const uint8_t* r, void* y, int64_t A, int64_t N, int64_t K, int32_t E, int tn,
+                                const void* tiles, const int32_t* num_tiles, const int32_t* sorted_rows,
+                                int max_tiles, int* status, cudaStream_t stream);
+
 // Grouped linear.
-size_t moe_workspace_bytes(int64_t A, int32_t E);
+size_t moe_workspace_bytes(int64_t A, int32_t E, int64_t K);
 cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const int32_t* token_of_row,
                        const int32_t* expert_of_row, const uint8_t* p, const uint8_t* r, void* y, int64_t A,
                        int64_t T, int64_t N, int64_t K, int32_t E, void* workspace, int* status,

@@ -1,11 +1,18 @@
-// Grouped (MoE) linear layer: device-side routing pre-pass + grouped kernels.
+// Grouped (MoE) linear layer: device-side routing pre-pass, activation gather, grouped kernel.
 // Paper: "Scheduler: Dual-Precision Execution", paragraph "Dual-mode serving (DPS) with
 // asymmetric switching" -- GroupedGEMM kernels with nested reconstruction serve MoE models.
 //
-// Workspace layout (int32 words, E4 = E rounded up to 4, A4 = A rounded up to 4):
-//   counts[E4] | offsets[E4 + 4] | sorted_rows[A4] | reserved
-// sorted_rows lists the valid row ids grouped by expert, in ascending row order inside each
-// group (a stable grouping, so the layout is reproducible).
+// Steps, all enqueued on the caller's stream without synchronising:
+//   1. route   (one CTA): validate rows, count rows per expert, group row ids by expert in
+//               ascending row order (stable, no atomics), and cut every group into token tiles.
+//   2. gather  : x_sorted[i][:] = x[token(sorted_rows[i])][:], so that each expert's activations
+//               are one contiguous matrix a TMA tile load can address.
+//   3. grouped tensor-core kernel over (weight-row tile, token tile): every expert's planes are
+//               streamed once per token tile; results are scattered to the caller's row order.
+//
+// Workspace layout (E4 = E rounded up to 4, A4 = A rounded up to 4, all parts 16-byte aligned):
+//   int32 counts[E4] | int32 offsets[E4 + 4] | int32 sorted_rows[A4] | int32 num_tiles[4]
+//   | int4 tiles[A4 / 16 + E + 4] | fp16 x_sorted[A][K]
 #include "dps_internal.h"
 #include "gemv.cuh"
 
@@ -16,11 +23,34 @@ namespace {
 constexpr int kRouteThreads = 1024;
 constexpr int kMaxExperts = 1024;
 
-struct EncMask {
-    uint32_t e5m2[kMaxExperts / 32];  // bit e set: expert e uses E5M2, else E4M3
+inline int64_t round4(int64_t v) { return (v + 3) / 4 * 4; }
+
+struct Workspace {
+    int32_t* counts;
+    int32_t* offsets;
+    int32_t* sorted_rows;
+    int32_t* num_tiles;
+    int4* tiles;
+    __half* x_sorted;
+    int64_t max_tiles;
+    size_t bytes;
 };
 
-inline int64_t round4(int64_t v) { return (v + 3) / 4 * 4; }
+Workspace carve(void* base, int64_t A, int32_t E, int64_t K) {
+    Workspace w;
+    const int64_t e4 = round4(E), a4 = round4(A);
+    int32_t* p = static_cast<int32_t*>(base);
+    w.counts = p;
+    w.offsets = w.counts + e4;
+    w.sorted_rows = w.offsets + e4 + 4;
+    w.num_tiles = w.sorted_rows + a4;
+    w.max_tiles = a4 / 16 + E + 4;
+    w.tiles = reinterpret_cast<int4*>(w.num_tiles + 4);
+    w.x_sorted = reinterpret_cast<__half*>(w.tiles + w.max_tiles);
+    const size_t head = (size_t)(e4 + e4 + 4 + a4 + 4) * 4 + (size_t)w.max_tiles * 16;
+    w.bytes = (head + (size_t)A * (size_t)K * 2 + 255) / 256 * 256;
+    return w;
+}
 
 __device__ __forceinline__ bool row_valid(const int32_t* token_of_row, const int32_t* expert_of_row, int a,
                                           int T, int E) {
@@ -34,7 +64,8 @@ __device__ __forceinline__ bool row_valid(const int32_t* token_of_row, const int
 // status word.
 __global__ void __launch_bounds__(kRouteThreads)
 moe_route_kernel(const int32_t* __restrict__ token_of_row, const int32_t* __restrict__ expert_of_row, int A, int T,
-                 int E, int32_t* counts, int32_t* offsets, int32_t* sorted_rows, int* status) {
+                 int E, int tile_tokens, int32_t* counts, int32_t* offsets, int32_t* sorted_rows,
+                 int32_t* num_tiles, int4* tiles, int* status) {
     __shared__ int s_cnt[kMaxExperts];
     __shared__ int s_off[kMaxExperts];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -52,14 +83,20 @@ moe_route_kernel(const int32_t* __restrict__ token_of_row, const int32_t* __rest
     }
     __syncthreads();
     if (tid == 0) {
-        int run = 0;
+        int run = 0, nt = 0;
         for (int e = 0; e < E; ++e) {
             s_off[e] = run;
             offsets[e] = run;
             counts[e] = s_cnt[e];
+            for (int first = 0; first < s_cnt[e]; first += tile_tokens) {
+                const int rows = s_cnt[e] - first < tile_tokens ? s_cnt[e] - first : tile_tokens;
+                tiles[nt++] = make_int4(e, run + first, rows, 0);
+            }
             run += s_cnt[e];
         }
         offsets[E] = run;
+        num_tiles[0] = nt;
+        num_tiles[1] = run;  // number of valid rows
     }
     __syncthreads();
     for (int e = warp; e < E; e += kRouteThreads / 32) {
@@ -74,92 +111,54 @@ moe_route_kernel(const int32_t* __restrict__ token_of_row, const int32_t* __rest
     }
 }
 
-// Interim grouped kernel on the CUDA-core GEMV body: blockIdx.y = expert, blockIdx.x = row
-// range of that expert's matrix; tokens of the group are taken four at a time.
-template <bool FULL>
-__global__ void __launch_bounds__(kGemvThreads, 2)
-moe_gemv_kernel(const __half* __restrict__ x, const int32_t* __restrict__ token_of_row,
-                const int32_t* __restrict__ sorted_rows, const int32_t* __restrict__ counts,
-                const int32_t* __restrict__ offsets, const uint8_t* __restrict__ P,
-                const uint8_t* __restrict__ Rp, __half* __restrict__ y, int64_t N, int64_t K, EncMask enc,
-                int rows_per_cta, int red_stride) {
-    extern __shared__ float red[];
-    const int e = blockIdx.y;
-    const int cnt = counts[e];
-    if (cnt == 0) return;
-    const int off = offsets[e];
-    const int64_t row_begin = (int64_t)blockIdx.x * rows_per_cta;
-    const int64_t row_end = (row_begin + rows_per_cta < N) ? row_begin + rows_per_cta : N;
-    if (row_begin >= row_end) return;
-    const uint8_t* Pe = P + (int64_t)e * N * K;
-    const uint8_t* Re = FULL ? Rp + (int64_t)e * N * K : nullptr;
-    const bool e5m2 = (enc.e5m2[e >> 5] >> (e & 31)) & 1u;
-    for (int g = 0; g < cnt; g += 4) {
-        const __half* xrow[4];
-        __half* yrow[4];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            xrow[t] = nullptr;
-            yrow[t] = nullptr;
-            if (g + t < cnt) {
-                const int a = sorted_rows[off + g + t];
-                const int tok = token_of_row ? token_of_row[a] : a;
-                xrow[t] = x + (int64_t)tok * K;
-                yrow[t] = y + (int64_t)a * N;
-            }
-        }
-        if (e5m2) gemv_rows<kEncE5M2, FULL, 4>(xrow, yrow, Pe, Re, K, row_begin, row_end, red, red_stride);
-        else gemv_rows<kEncE4M3, FULL, 4>(xrow, yrow, Pe, Re, K, row_begin, row_end, red, red_stride);
+// x_sorted[i][:] = x[token(sorted_rows[i])][:] for the valid rows; 16 bytes per thread.
+__global__ void __launch_bounds__(256)
+moe_gather_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ token_of_row,
+                  const int32_t* __restrict__ sorted_rows, const int32_t* __restrict__ num_tiles,
+                  uint4* __restrict__ x_sorted, int64_t k16) {
+    const int valid = num_tiles[1];
+    for (int i = blockIdx.x; i < valid; i += gridDim.x) {
+        const int a = sorted_rows[i];
+        const int64_t tok = token_of_row ? token_of_row[a] : a;
+        const uint4* src = x + tok * k16;
+        uint4* dst = x_sorted + (int64_t)i * k16;
+        for (int64_t c = threadIdx.x; c < k16; c += blockDim.x) dst[c] = src[c];
     }
 }
 
 }  // namespace
 
-size_t moe_workspace_bytes(int64_t A, int32_t E) {
-    if (A < 0 || E <= 0 || E > kMaxExperts || A > (int64_t)1 << 30) return 0;
-    const int64_t words = round4(E) + (round4(E) + 4) + round4(A);
-    const int64_t reserved = 16 * (A / 16 + E + 16);
-    return (size_t)((words * 4 + reserved + 255) / 256 * 256);
+size_t moe_workspace_bytes(int64_t A, int32_t E, int64_t K) {
+    if (A < 0 || E <= 0 || E > kMaxExperts || A > (int64_t)1 << 30 || K <= 0 || K > (int64_t)1 << 31) return 0;
+    return carve(nullptr, A, E, K).bytes;
 }
 
 cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const int32_t* token_of_row,
                        const int32_t* expert_of_row, const uint8_t* p, const uint8_t* r, void* y, int64_t A,
                        int64_t T, int64_t N, int64_t K, int32_t E, void* workspace, int* status,
                        cudaStream_t stream) {
-    int32_t* counts = static_cast<int32_t*>(workspace);
-    int32_t* offsets = counts + round4(E);
-    int32_t* sorted_rows = offsets + round4(E) + 4;
-    moe_route_kernel<<<1, kRouteThreads, 0, stream>>>(token_of_row, expert_of_row, (int)A, (int)T, E, counts, offsets,
-                                                      sorted_rows, status);
+    const Workspace w = carve(workspace, A, E, K);
+    const int tn = grouped_tile_tokens(A, E);
+    moe_route_kernel<<<1, kRouteThreads, 0, stream>>>(token_of_row, expert_of_row, (int)A, (int)T, E, tn, w.counts,
+                                                      w.offsets, w.sorted_rows, w.num_tiles, w.tiles, status);
     count_launch();
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-
-    EncMask enc;
-    for (int i = 0; i < kMaxExperts / 32; ++i) enc.e5m2[i] = 0;
-    for (int e = 0; e < E; ++e)
-        if (enc_host[e] == DPS_ENC_E5M2) enc.e5m2[e >> 5] |= 1u << (e & 31);
-
-    constexpr int MT = 4;
-    const int64_t max_rows = (32 * 1024) / (kGemvWarps * MT * 4) / kGemvRows * kGemvRows;
-    int64_t per_expert = ((int64_t)sm_count() * 2 + E - 1) / E;
-    int64_t rows = (N + per_expert - 1) / per_expert;
-    if (rows < 1) rows = 1;
-    if (rows > max_rows) rows = max_rows;
-    const int64_t gx = (N + rows - 1) / rows;
-    const int red_stride = (int)((rows + kGemvRows - 1) / kGemvRows) * kGemvRows * MT;
-    const size_t smem = (size_t)kGemvWarps * red_stride * sizeof(float);
-    dim3 grid((unsigned)gx, (unsigned)E);
-    const __half* xh = static_cast<const __half*>(x);
-    __half* yh = static_cast<__half*>(y);
-    if (mode == DPS_MODE_FULL)
-        moe_gemv_kernel<true><<<grid, kGemvThreads, smem, stream>>>(xh, token_of_row, sorted_rows, counts, offsets, p,
-                                                                    r, yh, N, K, enc, (int)rows, red_stride);
-    else
-        moe_gemv_kernel<false><<<grid, kGemvThreads, smem, stream>>>(xh, token_of_row, sorted_rows, counts, offsets,
-                                                                     p, r, yh, N, K, enc, (int)rows, red_stride);
+    const int gather_grid = (int)(A < 4096 ? A : 4096);
+    moe_gather_kernel<<<gather_grid, 256, 0, stream>>>(static_cast<const uint4*>(x), token_of_row, w.sorted_rows,
+                                                      w.num_tiles, reinterpret_cast<uint4*>(w.x_sorted), K / 8);
     count_launch();
-    return cudaGetLastError();
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+
+    uint32_t mask[kMaxExperts / 32];
+    for (int i = 0; i < kMaxExperts / 32; ++i) mask[i] = 0;
+    for (int e = 0; e < E; ++e)
+        if (enc_host[e] == DPS_ENC_E5M2) mask[e >> 5] |= 1u << (e & 31);
+    // an upper bound on the number of token tiles that needs no device round trip
+    const int max_tiles = (int)((A + tn - 1) / tn + E);
+    return launch_umma_grouped(mode, mask, w.x_sorted, p, r, y, A, N, K, E, tn, w.tiles, w.num_tiles, w.sorted_rows,
+                               max_tiles < w.max_tiles ? max_tiles : (int)w.max_tiles, status, stream);
 }
 
 }  // namespace dps

@@ -84,6 +84,15 @@ __device__ unsigned long long g_cta_times[2048 * 8];
 #define DPS_CTA_STAMP(ev) do { } while (0)
 #endif
 
+// Grouped (MoE) launches: blockIdx.y indexes a list of token tiles built on the device by the
+// routing pre-pass; each entry is (expert, first sorted row, rows in the tile, unused).
+struct GroupedParams {
+    const int4* tiles;
+    const int32_t* num_tiles;
+    const int32_t* sorted_rows;   // sorted position -> caller's row id
+    uint32_t e5m2[32];            // bit e set: expert e is E5M2
+};
+
 struct UmmaParams {
     __half* y;
     int M, N, K;
@@ -94,10 +103,72 @@ struct UmmaParams {
 
 };
 
-template <int ENC, bool FULL, int TN>
+// What a zip warp needs to know about its CTA's pipeline.
+struct ZipCtx {
+    int group, warp, lane, row, num_kb, num_stages, stage_bytes;
+    uint32_t smem_base, tmem_a, lane_base, sw;
+    uint64_t *bar_full, *bar_empty, *bar_a_full, *bar_a_empty;
+};
+
+// Zip loop of one warp: for each of its K blocks, wait for the planes to land and for the A slot
+// to be free, rebuild 128 FP16 weights of this thread's row from the plane bytes and store them
+// into tensor memory.  Returns false if a wait timed out.
+template <int ENC, bool FULL>
+__device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
+    bool ok = true;
+    for (int i = z.group; i < z.num_kb && ok; i += kZipGroups) {
+        const int s = i % z.num_stages, a = i % kAStages;
+        if (z.warp == 2 + 4 * z.group) DPS_STAMP(4, i);
+        ok = mbar_wait(smem_u32(&z.bar_full[s]), (uint32_t)(i / z.num_stages) & 1u);
+        if (z.warp == 2 + 4 * z.group) DPS_STAMP(5, i);
+        if (ok) ok = mbar_wait(smem_u32(&z.bar_a_empty[a]), ((uint32_t)(i / kAStages) & 1u) ^ 1u);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        if (z.warp == 2 + 4 * z.group) DPS_STAMP(6, i);
+        tc_fence_after_sync();
+        const uint32_t prow = z.smem_base + (uint32_t)s * z.stage_bytes + (uint32_t)z.row * kBlockK;
+        uint32_t h[kACols];
+#pragma unroll
+        for (int c = 0; c < kBlockK / 16; ++c) {
+            const uint32_t off = ((uint32_t)c ^ z.sw) * 16u;
+            uint4 pv, rv = make_uint4(0, 0, 0, 0);
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(pv.x), "=r"(pv.y), "=r"(pv.z), "=r"(pv.w)
+                         : "r"(prow + off));
+            if (FULL)
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(rv.x), "=r"(rv.y), "=r"(rv.z), "=r"(rv.w)
+                             : "r"(prow + kPlaneStageBytes + off));
+            uint32_t h8[8];
+            join16<ENC, FULL>(pv, rv, h8);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) h[c * 8 + j] = h8[j];
+        }
+#pragma unroll
+        for (int t = 0; t < kACols / 32; ++t) {
+            uint32_t part[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) part[j] = h[t * 32 + j];
+            tmem_st_32x32b_x32(z.tmem_a + z.lane_base + (uint32_t)(a * kACols + t * 32), part);
+        }
+        if (z.warp == 2 + 4 * z.group) DPS_STAMP(7, i);
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (z.lane == 0) {
+            mbar_arrive(smem_u32(&z.bar_a_full[a]));
+            mbar_arrive(smem_u32(&z.bar_empty[s]));
+        }
+        if (z.warp == 2 + 4 * z.group) DPS_STAMP(8, i);
+    }
+    return ok;
+}
+
+// ENC == 0 (grouped launches only): the encoding is a per-expert run-time value.
+template <int ENC, bool FULL, int TN, bool GROUPED>
 __global__ void __launch_bounds__(kThreads, (tmem_cols(TN) <= 256 ? 2 : 1))
 umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
-                   const __grid_constant__ CUtensorMap map_x, const UmmaParams prm) {
+                   const __grid_constant__ CUtensorMap map_x, const UmmaParams prm, const GroupedParams gp) {
     constexpr int kStage = stage_bytes(FULL, TN);
     constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
     constexpr uint32_t kCols = tmem_cols(TN);
@@ -125,7 +196,19 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_stages = prm.num_stages;
     const int n0 = blockIdx.x * kTileRows;
-    const int m0 = blockIdx.y * TN;
+    int m0 = blockIdx.y * TN;        // first token (dense) / first sorted row (grouped) of the tile
+    int tile_tokens = TN;            // valid token columns of the tile (grouped)
+    int plane_row0 = n0;             // first plane row of the tile in the [E * N][K] view
+    bool e5m2 = (ENC == kEncE5M2);
+    if (GROUPED) {
+        grid_dependency_wait();      // the tile list comes from the routing pre-pass
+        if ((int)blockIdx.y >= *gp.num_tiles) return;
+        const int4 t = gp.tiles[blockIdx.y];
+        m0 = t.y;
+        tile_tokens = t.z;
+        plane_row0 = t.x * prm.N + n0;
+        e5m2 = (gp.e5m2[t.x >> 5] >> (t.x & 31)) & 1u;
+    }
     const int total_kb = (prm.K + kBlockK - 1) / kBlockK;
     const int split = prm.split;
     const int rank = (split > 1) ? (int)cluster_ctarank() : 0;   // == blockIdx.z
@@ -191,8 +274,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 const uint32_t dst = smem_base + (uint32_t)s * kStage;
                 const int k = (rank + i * split) * kBlockK;
                 mbar_arrive_expect_tx(full, (uint32_t)kStage);
-                tma_load_2d(dst, &map_p, full, k, n0);
-                if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, n0);
+                tma_load_2d(dst, &map_p, full, k, plane_row0);
+                if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, plane_row0);
 #pragma unroll
                 for (int t = 0; t < kXAtoms; ++t)
                     tma_load_2d(dst + kXOffset + (uint32_t)(t * TN * 128), &map_x, full, k + t * 64, m0);
@@ -233,51 +316,17 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         const int q = warp & 3;                  // TMEM lane quarter this warp may touch
         const int row = q * 32 + lane;           // weight row inside the tile
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-        const uint32_t sw = (uint32_t)(row & 7);  // 128-byte swizzle: 16-byte chunk index ^= row % 8
-        for (int i = group; i < num_kb && ok; i += kZipGroups) {
-            const int s = i % num_stages, a = i % kAStages;
-            if (warp == 2 + 4 * group) DPS_STAMP(4, i);
-            ok = mbar_wait(smem_u32(&bar_full[s]), (uint32_t)(i / num_stages) & 1u);
-            if (warp == 2 + 4 * group) DPS_STAMP(5, i);
-            if (ok) ok = mbar_wait(smem_u32(&bar_a_empty[a]), ((uint32_t)(i / kAStages) & 1u) ^ 1u);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            if (warp == 2 + 4 * group) DPS_STAMP(6, i);
-            tc_fence_after_sync();
-            const uint32_t prow = smem_base + (uint32_t)s * kStage + (uint32_t)row * kBlockK;
-            uint32_t h[kACols];
-#pragma unroll
-            for (int c = 0; c < kBlockK / 16; ++c) {
-                const uint32_t off = ((uint32_t)c ^ sw) * 16u;
-                uint4 pv, rv = make_uint4(0, 0, 0, 0);
-                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                             : "=r"(pv.x), "=r"(pv.y), "=r"(pv.z), "=r"(pv.w)
-                             : "r"(prow + off));
-                if (FULL)
-                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                                 : "=r"(rv.x), "=r"(rv.y), "=r"(rv.z), "=r"(rv.w)
-                                 : "r"(prow + kPlaneStageBytes + off));
-                uint32_t h8[8];
-                join16<ENC, FULL>(pv, rv, h8);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) h[c * 8 + j] = h8[j];
-            }
-#pragma unroll
-            for (int t = 0; t < kACols / 32; ++t) {
-                uint32_t part[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) part[j] = h[t * 32 + j];
-                tmem_st_32x32b_x32(tmem_a + lane_base + (uint32_t)(a * kACols + t * 32), part);
-            }
-            if (warp == 2 + 4 * group) DPS_STAMP(7, i);
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(smem_u32(&bar_a_full[a]));
-                mbar_arrive(smem_u32(&bar_empty[s]));
-            }
-            if (warp == 2 + 4 * group) DPS_STAMP(8, i);
+        ZipCtx zc;
+        zc.group = group; zc.warp = warp; zc.lane = lane; zc.row = row;
+        zc.num_kb = num_kb; zc.num_stages = num_stages; zc.stage_bytes = kStage;
+        zc.smem_base = smem_base; zc.tmem_a = tmem_a; zc.lane_base = lane_base;
+        zc.sw = (uint32_t)(row & 7);  // 128-byte swizzle: 16-byte chunk index ^= row % 8
+        zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
+        if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2)) {
+            // encoding known only at run time (one per expert): uniform branch per CTA
+            ok = e5m2 ? zip_blocks<kEncE5M2, FULL>(zc) : zip_blocks<kEncE4M3, FULL>(zc);
+        } else {
+            ok = zip_blocks<ENC, FULL>(zc);
         }
         // epilogue (first zip group): D[row][token] -> y[token][n0 + row], or -> red for split K
         if (group == 0) {
@@ -305,8 +354,13 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                     } else if (n < prm.N) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
-                            const int m = m0 + c0 + j;
-                            if (m < prm.M) prm.y[(int64_t)m * prm.N + n] = __float2half_rn(__uint_as_float(v[j]));
+                            int m = m0 + c0 + j;
+                            bool valid = m < prm.M;
+                            if (GROUPED) {
+                                valid = (c0 + j) < tile_tokens;
+                                if (valid) m = gp.sorted_rows[m];
+                            }
+                            if (valid) prm.y[(int64_t)m * prm.N + n] = __float2half_rn(__uint_as_float(v[j]));
                         }
                     }
                 }
@@ -424,7 +478,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     stages -= stages % kZipGroups;  // a stage always belongs to the same zip group, so that every
                                     // waiter sees every phase of the barriers it waits on
     const size_t smem = (size_t)stages * kStage + kMailBytes + 1024;
-    auto kernel = umma_linear_kernel<ENC, FULL, TN>;
+    auto kernel = umma_linear_kernel<ENC, FULL, TN, false>;
     static int capacity[kMaxSplit + 1] = {0};  // per instantiation; filled on first use
     static bool configured = false;
     if (!configured) {
@@ -512,7 +566,8 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, prm);
+    GroupedParams gp = {};
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, prm, gp);
     count_launch();
     return e;
 }
@@ -538,6 +593,101 @@ extern "C" __attribute__((visibility("default"))) int dps_debug_cta_times(unsign
     return (int)cudaMemcpyFromSymbol(out, g_cta_times, sizeof(unsigned long long) * 2048 * 8);
 }
 #endif
+
+namespace {
+
+template <bool FULL, int TN>
+cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, const uint8_t* p, const uint8_t* r,
+                              void* y, int64_t A, int64_t N, int64_t K, int32_t E, const void* tiles,
+                              const int32_t* num_tiles, const int32_t* sorted_rows, int max_tiles, int* status,
+                              cudaStream_t stream) {
+    constexpr int kStage = stage_bytes(FULL, TN);
+    constexpr int kCtasPerSm = tmem_cols(TN) <= 256 ? 2 : 1;
+    constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
+    int stages = kSmemTotal / kStage;
+    if (stages > 8) stages = 8;
+    if (stages < 2) stages = 2;
+    stages -= stages % kZipGroups;
+    const size_t smem = (size_t)stages * kStage + 1024;
+    auto kernel = umma_linear_kernel<0, FULL, TN, true>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    CUtensorMap mp, mr, mx;
+    if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows,
+                     kBlockK, CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
+    if (FULL) {
+        if (!make_map_2d(&mr, r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows,
+                         kBlockK, CU_TENSOR_MAP_SWIZZLE_128B))
+            return cudaErrorInvalidValue;
+    } else {
+        mr = mp;
+    }
+    if (!make_map_2d(&mx, x_sorted, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)A, (uint64_t)K, TN, 64,
+                     CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
+    UmmaParams prm;
+    prm.y = static_cast<__half*>(y);
+    prm.M = (int)A;
+    prm.N = (int)N;
+    prm.K = (int)K;
+    prm.num_stages = stages;
+    prm.split = 1;
+    prm.red_offset = 0;
+    prm.status = status;
+    GroupedParams gp;
+    gp.tiles = static_cast<const int4*>(tiles);
+    gp.num_tiles = num_tiles;
+    gp.sorted_rows = sorted_rows;
+    for (int i = 0; i < 32; ++i) gp.e5m2[i] = e5m2_mask[i];
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((N + kTileRows - 1) / kTileRows), (unsigned)max_tiles, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, prm, gp);
+    count_launch();
+    return e;
+}
+
+}  // namespace
+
+int grouped_tile_tokens(int64_t A, int32_t E) {
+    const int64_t target = 2 * ((A + E - 1) / E);
+    return target <= 16 ? 16 : target <= 32 ? 32 : target <= 64 ? 64 : 128;
+}
+
+cudaError_t launch_umma_grouped(int mode, const uint32_t* e5m2_mask, const void* x_sorted, const uint8_t* p,
+                                const uint8_t* r, void* y, int64_t A, int64_t N, int64_t K, int32_t E, int tn,
+                                const void* tiles, const int32_t* num_tiles, const int32_t* sorted_rows,
+                                int max_tiles, int* status, cudaStream_t stream) {
+#define DPS_GROUPED_CASE(TNV)                                                                                     \
+    if (tn == TNV)                                                                                                \
+        return mode == DPS_MODE_FULL                                                                              \
+                   ? launch_grouped_tn<true, TNV>(e5m2_mask, x_sorted, p, r, y, A, N, K, E, tiles, num_tiles,     \
+                                                  sorted_rows, max_tiles, status, stream)                        \
+                   : launch_grouped_tn<false, TNV>(e5m2_mask, x_sorted, p, r, y, A, N, K, E, tiles, num_tiles,    \
+                                                   sorted_rows, max_tiles, status, stream);
+    DPS_GROUPED_CASE(16)
+    DPS_GROUPED_CASE(32)
+    DPS_GROUPED_CASE(64)
+    DPS_GROUPED_CASE(128)
+#undef DPS_GROUPED_CASE
+    return cudaErrorInvalidValue;
+}
 
 cudaError_t launch_umma_linear(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
                                int64_t M, int64_t N, int64_t K, int* status, cudaStream_t stream) {

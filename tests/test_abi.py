@@ -35,11 +35,13 @@ def test_version_and_status_strings():
 
 
 def test_workspace_size_function():
-    assert binding.dps_moe_workspace_bytes(512, 8) >= 4 * (512 + 2 * 8 + 1)
-    assert binding.dps_moe_workspace_bytes(0, 8) > 0
-    assert binding.dps_moe_workspace_bytes(-1, 8) == 0
-    assert binding.dps_moe_workspace_bytes(16, 0) == 0
-    assert binding.dps_moe_workspace_bytes(1 << 20, 64) % 256 == 0
+    assert binding.dps_moe_workspace_bytes(512, 8, 4096) >= 4 * (512 + 2 * 8 + 1) + 512 * 4096 * 2
+    assert binding.dps_moe_workspace_bytes(0, 8, 64) > 0
+    assert binding.dps_moe_workspace_bytes(-1, 8, 64) == 0
+    assert binding.dps_moe_workspace_bytes(16, 0, 64) == 0
+    assert binding.dps_moe_workspace_bytes(16, 2000, 64) == 0
+    assert binding.dps_moe_workspace_bytes(16, 8, 0) == 0
+    assert binding.dps_moe_workspace_bytes(1 << 20, 64, 1024) % 256 == 0
 
 
 def test_host_validation_needs_no_device():
@@ -79,7 +81,7 @@ def test_host_validation_needs_no_device():
     encs = (ctypes.c_int32 * 2)(1, 2)
     bad = (ctypes.c_int32 * 2)(1, 0)
     args = dict(A=4, T=4, N=8, K=16, E=2)
-    def moe(mode=0, enc=encs, x=fake, tor=None, eor=fake, p=fake, r=None, y=fake, ws=fake, wsb=1 << 20, **kw):
+    def moe(mode=0, enc=encs, x=fake, tor=None, eor=fake, p=fake, r=None, y=fake, ws=fake, wsb=1 << 24, **kw):
         a = {**args, **kw}
         return lib.dps_moe_linear(mode, enc, x, tor, eor, p, r, y, a["A"], a["T"], a["N"], a["K"], a["E"], ws, wsb, None)
     assert moe(mode=5) == binding.DPS_ERR_MODE
