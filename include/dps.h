@@ -134,6 +134,39 @@ DPS_API dps_status dps_moe_linear(int32_t mode, const int32_t* enc_per_expert, c
 DPS_API size_t dps_moe_workspace_bytes(int64_t A, int32_t E, int64_t K);
 
 /*
+ * Grouped linear layer for callers that cannot allocate (the paper has no counterpart; this is a
+ * convenience of this library).
+ *
+ * Some callers have no way to hand dps_moe_linear a workspace: a serving worker that gave all of
+ * its free device memory to the weight planes and the KV cache at start-up and runs its steps under
+ * a rule that nothing may call cudaMalloc afterwards (an allocation there synchronises the device,
+ * can fail when memory is fully committed, and is forbidden outright in some runtimes), or a
+ * plug-in that is only ever given its input and output buffers.  For them this variant computes
+ * exactly what dps_moe_linear computes, with the same kernels, but keeps its scratch (routing tables
+ * and the activations regrouped by expert) in a fixed array inside the library instead of a caller
+ * buffer.  The call itself allocates nothing and frees nothing.
+ *
+ * Limits and rules:
+ *   - The array is DPS_MOE_STATIC_SCRATCH_BYTES (16 MiB) per GPU and is held by every GPU that loads
+ *     the library until the process exits.  A problem whose dps_moe_workspace_bytes(A, E, K) exceeds
+ *     it is rejected with DPS_ERR_WORKSPACE and nothing is enqueued; use dps_moe_linear then.
+ *   - The first call on each device looks up the array's device address (a one-time, host-side
+ *     set-up step).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left in it.
+ *     Nothing in it has to start at zero: every call rewrites all the tables it reads.  Two calls
+ *     whose kernels can overlap on the GPU (different streams without an ordering between them)
+ *     would overwrite each other's scratch: keep calls on one stream or order them with events.
+ * Arguments, layouts, error codes and the status word are those of dps_moe_linear, minus the
+ * workspace pair.  Never synchronises.
+ */
+#define DPS_MOE_STATIC_SCRATCH_BYTES (16u << 20)
+DPS_API dps_status dps_moe_linear_static(int32_t mode, const int32_t* enc_per_expert, const void* x,
+                                         const int32_t* token_of_row, const int32_t* expert_of_row,
+                                         const uint8_t* w_persist, const uint8_t* w_resid, void* y,
+                                         int64_t A, int64_t T, int64_t N, int64_t K, int32_t E,
+                                         void* cuda_stream);
+
+/*
  * Synchronises the stream, then returns and clears the current device's status word:
  * DPS_OK, DPS_ERR_DATA (a kernel skipped a row with a bad index) or DPS_ERR_CUDA.
  */

@@ -28,6 +28,8 @@ ABI = {
     "dps_linear": (ctypes.c_int, [_i32, _i32, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "dps_moe_linear": (ctypes.c_int, [_i32, ctypes.POINTER(_i32), _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64,
                                       _i64, _i32, _vp, ctypes.c_size_t, _vp]),
+    "dps_moe_linear_static": (ctypes.c_int, [_i32, ctypes.POINTER(_i32), _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64,
+                                             _i64, _i32, _vp]),
     "dps_moe_workspace_bytes": (ctypes.c_size_t, [_i64, _i32, _i64]),
     "dps_stream_status": (ctypes.c_int, [_vp]),
     "dps_launch_count": (_i64, []),
@@ -159,6 +161,33 @@ def dps_moe_linear(mode: int, enc_per_expert: Sequence[int], x: torch.Tensor, to
                                   _dev(y, torch.float16, "y"), A, T, N, K, E,
                                   _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream))
     _check(st, "dps_moe_linear")
+    return y
+
+
+DPS_MOE_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def dps_moe_linear_static(mode: int, enc_per_expert: Sequence[int], x: torch.Tensor,
+                          token_of_row: Optional[torch.Tensor], expert_of_row: torch.Tensor,
+                          w_persist: torch.Tensor, w_resid: Optional[torch.Tensor], y: torch.Tensor,
+                          stream=None) -> torch.Tensor:
+    """Grouped linear for callers that must not allocate: same result as dps_moe_linear, scratch
+    kept in a fixed 16 MiB array inside the library.  The caller passes inputs and the output
+    tensor; nothing is allocated here either.  Problems that need more scratch raise DpsError
+    (DPS_ERR_WORKSPACE).  Calls share the array, so keep them ordered on the GPU."""
+    E, N, K = w_persist.shape
+    T, K2 = x.shape
+    if K != K2:
+        raise ValueError(f"K mismatch: x has {K}, planes have {K2}")
+    A = expert_of_row.numel()
+    enc_arr = (_i32 * E)(*[int(e) for e in enc_per_expert])
+    st = library().dps_moe_linear_static(int(mode), enc_arr, _dev(x, torch.float16, "x"),
+                                         _dev(token_of_row, torch.int32, "token_of_row"),
+                                         _dev(expert_of_row, torch.int32, "expert_of_row"),
+                                         _dev(w_persist, torch.uint8, "w_persist"),
+                                         _dev(w_resid, torch.uint8, "w_resid"), _dev(y, torch.float16, "y"), A, T,
+                                         N, K, E, _stream(stream))
+    _check(st, "dps_moe_linear_static")
     return y
 
 

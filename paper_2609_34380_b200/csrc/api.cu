@@ -69,6 +69,13 @@ dps_status check_device(DeviceInfo*& d) {
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+dps_status device_status_word(int** status) {
+    DeviceInfo* d = nullptr;
+    const dps_status st = check_device(d);
+    *status = (st == DPS_OK) ? d->status : nullptr;
+    return st;
+}
+
 int sm_count() {
     DeviceInfo* d = device_info();
     return (d && d->sms > 0) ? d->sms : 148;

@@ -42,6 +42,9 @@ cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const i
                        int64_t T, int64_t N, int64_t K, int32_t E, void* workspace, int* status,
                        cudaStream_t stream);
 
+// Checks that the current device can run the kernels and returns the address of its status word.
+dps_status device_status_word(int** status);
+
 void count_launch(int n = 1);
 int sm_count();
 

@@ -13,6 +13,8 @@
 // Workspace layout (E4 = E rounded up to 4, A4 = A rounded up to 4, all parts 16-byte aligned):
 //   int32 counts[E4] | int32 offsets[E4 + 4] | int32 sorted_rows[A4] | int32 num_tiles[4]
 //   | int4 tiles[A4 / 16 + E + 4] | fp16 x_sorted[A][K]
+#include <mutex>
+
 #include "dps_internal.h"
 #include "gemv.cuh"
 
@@ -162,3 +164,73 @@ cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const i
 }
 
 }  // namespace dps
+
+// ---- allocation-free variant ---------------------------------------------------------------------
+// Scratch for dps_moe_linear_static: one fixed array per GPU that loads the library, held until the
+// process exits.  In host code the array's name is only a stand-in; the device address is looked up
+// once per device (with that device current) and handed to the kernels as an ordinary pointer.
+namespace dps {
+namespace {
+
+constexpr size_t kStaticScratchBytes = (size_t)DPS_MOE_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_moe_static_scratch[kStaticScratchBytes];
+
+struct StaticScratch {
+    std::once_flag once;
+    cudaError_t err = cudaSuccess;
+    unsigned char* ptr = nullptr;
+};
+StaticScratch g_static_scratch[64];
+
+cudaError_t static_scratch_address(unsigned char** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    StaticScratch& s = g_static_scratch[dev];
+    std::call_once(s.once, [&] {
+        unsigned char* ptr = nullptr;
+        s.err = cudaGetSymbolAddress((void**)&ptr, g_moe_static_scratch);
+        s.ptr = (s.err == cudaSuccess) ? ptr : nullptr;
+    });
+    *out = s.ptr;
+    return s.err;
+}
+
+}  // namespace
+}  // namespace dps
+
+extern "C" DPS_API dps_status dps_moe_linear_static(int32_t mode, const int32_t* enc_per_expert, const void* x,
+                                                    const int32_t* token_of_row, const int32_t* expert_of_row,
+                                                    const uint8_t* w_persist, const uint8_t* w_resid, void* y,
+                                                    int64_t A, int64_t T, int64_t N, int64_t K, int32_t E,
+                                                    void* cuda_stream) {
+    using namespace dps;
+    if (mode != DPS_MODE_FAST && mode != DPS_MODE_FULL) return DPS_ERR_MODE;
+    if (A < 0 || T < 0 || N <= 0 || K <= 0 || E <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
+    if (A > ((int64_t)1 << 30) || T > ((int64_t)1 << 30) || N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31))
+        return DPS_ERR_SHAPE;
+    if (!enc_per_expert) return DPS_ERR_NULL;
+    const size_t need = moe_workspace_bytes(A, E, K);
+    if (need == 0) return DPS_ERR_SHAPE;
+    if (need > kStaticScratchBytes) return DPS_ERR_WORKSPACE;  // beyond the built-in scratch: use dps_moe_linear
+    for (int32_t e = 0; e < E; ++e)
+        if (enc_per_expert[e] != DPS_ENC_E4M3 && enc_per_expert[e] != DPS_ENC_E5M2) return DPS_ERR_ENCODING;
+    if (A == 0) return DPS_OK;
+    if (!x || !expert_of_row || !w_persist || !y) return DPS_ERR_NULL;
+    if (mode == DPS_MODE_FULL && !w_resid) return DPS_ERR_NULL;
+    auto misaligned = [](const void* p, uintptr_t mask) { return (reinterpret_cast<uintptr_t>(p) & mask) != 0; };
+    if (misaligned(x, 15) || misaligned(w_persist, 15) || misaligned(y, 15)) return DPS_ERR_ALIGN;
+    if (mode == DPS_MODE_FULL && misaligned(w_resid, 15)) return DPS_ERR_ALIGN;
+    if (misaligned(expert_of_row, 3) || misaligned(token_of_row, 3)) return DPS_ERR_ALIGN;
+    int* status = nullptr;
+    const dps_status st = device_status_word(&status);
+    if (st != DPS_OK) return st;
+    unsigned char* scratch = nullptr;
+    if (static_scratch_address(&scratch) != cudaSuccess || scratch == nullptr) return DPS_ERR_CUDA;
+    const uint8_t* r = (mode == DPS_MODE_FULL) ? w_resid : nullptr;
+    if (launch_moe(mode, enc_per_expert, x, token_of_row, expert_of_row, w_persist, r, y, A, T, N, K, E, scratch,
+                   status, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return DPS_ERR_CUDA;
+    return DPS_OK;
+}
