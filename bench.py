@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--copies", type=int, default=32, help="distinct weight copies per linear (L2 rotation)")
     ap.add_argument("--skip-detail", action="store_true", help="skip the extra rows (split, prefill, MoE)")
-    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="time budget of the CPU oracle sample")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="time budget of the CPU oracle sample")
     return ap.parse_args()
 
 
@@ -128,30 +128,35 @@ def linear_bytes(mode_full: bool, m: int, n: int, k: int) -> int:
 
 
 def oracle_sample(budget_s: float, threads: int):
-    """Runs the oracle as it stands on Llama-7B-shaped linears at M=1, both modes, smallest
-    layer first, until the time budget is used.  Returns (GB/s, description, seconds)."""
+    """Runs the oracle as it stands over the step's work list on ONE weight copy (layers smallest
+    first, then M, then mode) until the time budget is used.  Returns (GB/s, description, seconds)."""
     import numpy as np
     import oracle
     from paper_2609_34380_b200 import workloads
 
     order = ["o", "down", "qkv", "gate_up"]
+    planes = {}
+    rng = np.random.default_rng(2001)
     done, total_bytes, total_s = [], 0, 0.0
-    for name in order:
-        n, k = workloads.LLAMA7B[name]
-        if done and total_s > budget_s * 0.6:
-            break
-        rng = np.random.default_rng(2001)
-        w = (rng.standard_normal((n, k), dtype=np.float32) * 0.02).astype(np.float16)
-        x = rng.standard_normal((1, k), dtype=np.float32).astype(np.float16)
-        p, r, enc = oracle.split(w, oracle.ENC_AUTO)
-        for mode in (oracle.MODE_FAST, oracle.MODE_FULL):
-            t0 = time.perf_counter()
-            oracle.linear(mode, enc, x, p, r if mode else None, threads=threads)
-            total_s += time.perf_counter() - t0
-            total_bytes += linear_bytes(bool(mode), 1, n, k)
-        done.append(name)
+    for M in workloads.DECODE_M:
+        for name in order:
+            n, k = workloads.LLAMA7B[name]
+            if total_s > budget_s:
+                break
+            if name not in planes:
+                w = (rng.standard_normal((n, k), dtype=np.float32) * 0.02).astype(np.float16)
+                planes[name] = oracle.split(w, oracle.ENC_AUTO)
+            p, r, enc = planes[name]
+            x = rng.standard_normal((M, k), dtype=np.float32).astype(np.float16)
+            for mode in (oracle.MODE_FAST, oracle.MODE_FULL):
+                t0 = time.perf_counter()
+                oracle.linear(mode, enc, x, p, r if mode else None, threads=threads)
+                total_s += time.perf_counter() - t0
+                total_bytes += linear_bytes(bool(mode), M, n, k)
+            done.append(f"{name}@M{M}")
     gbs = total_bytes / total_s / 1e9
-    return gbs, f"oracle.linear (FP64, {threads} threads) on Llama-7B linears {done} at M=1, fast+full", total_s
+    return gbs, (f"oracle.linear (FP64 accumulate, {threads} threads), one weight copy of the step's work list, "
+                 f"fast+full: {','.join(done)}"), total_s
 
 
 def run_reference(args, rank: int):
@@ -325,6 +330,11 @@ def run_ours(args, rank: int, local_rank: int, world: int):
             "frac_of_nominal_8TBs": (b / (ms * 1e-3) / 1e9) / NOMINAL_HBM_GBS, "frac_of_roofline": t_roof / (ms * 1e-3),
             "us_per_layer_set": 1e3 * ms / copies}
 
+    if not args.skip_detail and world == 1:
+        del graphs, planes
+        torch.cuda.empty_cache()
+        detail.update(detail_rows(dps, workloads, torch, dev, peaks))
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -355,6 +365,157 @@ def run_ours(args, rank: int, local_rank: int, world: int):
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def _time_graph(torch, stream, enqueue, iters=5, warm=2):
+    """Median per-replay milliseconds of a CUDA graph holding enqueue()'s launches."""
+    with torch.cuda.stream(stream):
+        enqueue()
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            enqueue()
+        for _ in range(warm):
+            g.replay()
+        times = []
+        for _ in range(iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+    return statistics.median(times), g
+
+
+def detail_rows(dps, workloads, torch, dev, peaks):
+    """The other rows of the path, each timed on its own: split / reconstruct (load time), prefill
+    linears (config 3), grouped MoE linears (config 4) and the 32-layer decoder step under the
+    bursty mode schedule (config 5).  Reported beside the headline, never mixed into it."""
+    out = {}
+    stream = torch.cuda.Stream(device=dev)
+    hbm, tc = peaks["hbm_gbs"], peaks["bf16_tflops"]
+
+    # ---- split / reconstruct: 8 gate+up-shaped tensors (1.4 GB of FP16, larger than L2) ----
+    n, k = workloads.LLAMA7B["gate_up"]
+    ws = [workloads.weights(n, k, 2003 + 100 * c, device=dev) for c in range(8)]
+    P = torch.empty((8, n, k), dtype=torch.uint8, device=dev)
+    R = torch.empty((8, n, k), dtype=torch.uint8, device=dev)
+    W2 = torch.empty((8, n, k), dtype=torch.float16, device=dev)
+    ms, _ = _time_graph(torch, stream, lambda: [dps.dps_split_weights(ws[c], dps.DPS_ENC_E5M2, P[c], R[c]) for c in range(8)])
+    out["split"] = {"GB/s": 8 * n * k * 4 / (ms * 1e-3) / 1e9, "frac_of_measured_hbm": 8 * n * k * 4 / (ms * 1e-3) / 1e9 / hbm}
+    ms, _ = _time_graph(torch, stream, lambda: [dps.dps_reconstruct(P[c], R[c], dps.DPS_ENC_E5M2, W2[c]) for c in range(8)])
+    out["reconstruct"] = {"GB/s": 8 * n * k * 4 / (ms * 1e-3) / 1e9, "frac_of_measured_hbm": 8 * n * k * 4 / (ms * 1e-3) / 1e9 / hbm}
+    del ws, P, R, W2
+
+    # ---- prefill (config 3): 4 weight copies in rotation ----
+    pre = {}
+    planes = {name: [dps.dps_split_weights(workloads.weights(n, k, 2001 + i + 100 * c, device=dev), dps.DPS_ENC_AUTO)
+                     for c in range(4)] for i, (name, (n, k)) in enumerate(workloads.LLAMA7B.items())}
+    for M in workloads.PREFILL_M:
+        xs = {name: workloads.activations(M, k, 3001 + i, device=dev) for i, (name, (n, k)) in enumerate(workloads.LLAMA7B.items())}
+        ys = {name: torch.empty((M, n), dtype=torch.float16, device=dev) for name, (n, k) in workloads.LLAMA7B.items()}
+        for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):
+            def enqueue():
+                for c in range(4):
+                    for name in workloads.LLAMA7B:
+                        p, r, enc = planes[name][c]
+                        dps.dps_linear(mode, enc, xs[name], p, r if mode else None, ys[name])
+            ms, _ = _time_graph(torch, stream, enqueue, iters=3, warm=1)
+            flops = 4 * sum(2 * M * n * k for n, k in workloads.LLAMA7B.values())
+            tf = flops / (ms * 1e-3) / 1e12
+            pre[f"M{M}_{'full' if mode else 'fast'}"] = {"TFLOP/s": tf, "frac_of_measured_bf16_burst": tf / tc,
+                                                        "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
+                                                        "ms_per_layer_set": ms / 4}
+        del xs, ys
+    out["prefill"] = pre
+    del planes
+    torch.cuda.empty_cache()
+
+    # ---- MoE (config 4) ----
+    moe = {}
+    E, T = workloads.MIXTRAL_EXPERTS, workloads.MIXTRAL_TOKENS
+    tor, eor = workloads.top2_routing(T, E, 4200)
+    eor_d, tor_d = torch.from_numpy(eor).to(dev), torch.from_numpy(tor).to(dev)
+    used = len(set(eor.tolist()))
+    for li, (name, (n, k)) in enumerate(workloads.MIXTRAL_EXPERT.items()):
+        P = torch.empty((2, E, n, k), dtype=torch.uint8, device=dev)     # two copies: 1.9 / 0.9 GB per plane set
+        R = torch.empty((2, E, n, k), dtype=torch.uint8, device=dev)
+        encs = []
+        for c in range(2):
+            for e in range(E):
+                w = workloads.weights(n, k, 4001 + 10 * li + e + 100 * c, device=dev)
+                _, _, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO, P[c, e], R[c, e])
+                if c == 0:
+                    encs.append(enc)
+                del w
+        x = workloads.activations(T if name == "gate_up" else 2 * T, k, 4100 + li, device=dev)
+        tmap = tor_d if name == "gate_up" else None
+        y = torch.empty((2 * T, n), dtype=torch.float16, device=dev)
+        wsb = torch.empty(dps.dps_moe_workspace_bytes(2 * T, E, k), dtype=torch.uint8, device=dev)
+        for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):
+            ms, _ = _time_graph(torch, stream, lambda: [dps.dps_moe_linear(mode, encs, x, tmap, eor_d, P[c], R[c] if mode else None, y, wsb)
+                                                        for c in range(2)], iters=5, warm=1)
+            nbytes = 2 * (used * n * k * (2 if mode else 1) + x.numel() * 2 + y.numel() * 2)
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            moe[f"{name}_{'full' if mode else 'fast'}"] = {"GB/s": gbs, "frac_of_measured_hbm": gbs / hbm, "us_per_call": 1e3 * ms / 2}
+        del P, R, x, y, wsb
+    out["moe"] = moe
+    torch.cuda.empty_cache()
+
+    # ---- 32-layer decoder step under the bursty schedule (config 5) ----
+    layers = workloads.DECODER70_LAYERS
+    shapes = workloads.DECODER70
+    planes = []
+    for layer in range(layers):
+        row = {}
+        for i, (name, (n, k)) in enumerate(shapes.items()):
+            w = workloads.weights(n, k, 5000 + layer * 4 + i, device=dev)
+            row[name] = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+            del w
+        planes.append(row)
+    schedule = workloads.mode_schedule(256, 5555)
+    step_rows = {}
+    for M in workloads.STEP_M:
+        xs = {name: workloads.activations(M, k, 5901 + i, device=dev) for i, (name, (n, k)) in enumerate(shapes.items())}
+        ys = {name: torch.empty((M, n), dtype=torch.float16, device=dev) for name, (n, k) in shapes.items()}
+        graphs = {}
+        with torch.cuda.stream(stream):
+            for mode in (0, 1):
+                def enqueue():
+                    for row in planes:
+                        for name, (p, r, enc) in row.items():
+                            dps.dps_linear(mode, enc, xs[name], p, r if mode else None, ys[name])
+                enqueue()
+                stream.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    enqueue()
+                graphs[mode] = g
+            evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(schedule) + 1)]
+            for t, mode in enumerate(schedule):
+                evs[t].record(stream)
+                graphs[mode].replay()
+            evs[-1].record(stream)
+            stream.synchronize()
+        per = [evs[t].elapsed_time(evs[t + 1]) for t in range(len(schedule))]
+        row = {}
+        for mode, label in ((0, "fast"), (1, "full")):
+            steady = [per[t] for t in range(1, len(schedule)) if schedule[t] == mode and schedule[t - 1] == mode]
+            after = [per[t] for t in range(1, len(schedule)) if schedule[t] == mode and schedule[t - 1] != mode]
+            nbytes = layers * sum(linear_bytes(bool(mode), M, n, k) for n, k in shapes.values())
+            flops = layers * sum(2 * M * n * k for n, k in shapes.values())
+            t_roof = max(nbytes / (hbm * 1e9), flops / (tc * 1e12)) * 1e3
+            med = statistics.median(steady)
+            row[label] = {"ms_per_step": med, "GB/s": nbytes / (med * 1e-3) / 1e9, "TFLOP/s": flops / (med * 1e-3) / 1e12,
+                          "frac_of_roofline": t_roof / med,
+                          "ms_first_step_after_switch": statistics.median(after) if after else None}
+        step_rows[f"M{M}"] = row
+        del xs, ys, graphs
+    out["decoder_step_32_layers"] = {"schedule": {"steps": len(schedule), "fast_share": schedule.count(0) / len(schedule),
+                                                  "switches": sum(1 for i in range(1, len(schedule)) if schedule[i] != schedule[i - 1])},
+                                     "per_M": step_rows}
+    return out
 
 
 def main():

@@ -62,7 +62,7 @@ def main() -> None:
     us = 1e3 * start.elapsed_time(stop) / args.copies
     nbytes = n * k * (2 if mode else 1) + 2 * args.M * (n + k)
     print(f"{args.family}/{args.layer} N={n} K={k} M={args.M} {args.mode}: {us:.2f} us/launch, "
-          f"{nbytes / us / 1e3:.0f} GB/s, status={dps.dps_stream_status()}")
+          f"{nbytes / us / 1e3:.0f} GB/s, {2 * args.M * n * k / us / 1e6:.1f} TFLOP/s, status={dps.dps_stream_status()}")
 
 
 if __name__ == "__main__":
