@@ -44,13 +44,14 @@ DeviceInfo* device_info() {
     return &d;
 }
 
-// Tuning / debugging knob: DPS_FORCE_PATH=gemv or =umma pins the dense kernel family.
+// Tuning / debugging knob: DPS_FORCE_PATH=gemv, =umma or =stream pins the dense kernel family.
 int forced_path() {
     static const int path = [] {
         const char* v = getenv("DPS_FORCE_PATH");
         if (!v) return 0;
         if (!strcmp(v, "gemv")) return 1;
         if (!strcmp(v, "umma")) return 2;
+        if (!strcmp(v, "stream")) return 3;
         return 0;
     }();
     return path;
@@ -162,12 +163,16 @@ dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w
     if (st != DPS_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const uint8_t* r = (mode == DPS_MODE_FULL) ? w_resid : nullptr;  // fast mode never sees the pointer
-    // Up to four tokens the CUDA-core GEMV wins (no tensor-memory set-up, exact FP32 FMAs keep up
-    // with the weight stream); beyond that the tensor cores take the arithmetic.
+    // Up to 16 tokens the layer is a pure weight stream: the register-streaming kernel serves it.
+    // Beyond that the tcgen05 tiles take over.  (The CUDA-core GEMV is kept as a cross-check.)
     const int path = forced_path();
-    const bool use_gemv = path == 1 || (path == 0 && M <= 4);
-    cudaError_t err = use_gemv ? launch_gemv(mode, enc, x, w_persist, r, y, M, N, K, stream)
-                               : launch_umma_linear(mode, enc, x, w_persist, r, y, M, N, K, d->status, stream);
+    cudaError_t err;
+    if (path == 1) err = launch_gemv(mode, enc, x, w_persist, r, y, M, N, K, stream);
+    else if (path == 2) err = launch_umma_linear(mode, enc, x, w_persist, r, y, M, N, K, d->status, stream);
+    else if (path == 3 || M <= 16) {
+        if (M > 16) return DPS_ERR_UNSUPPORTED;
+        err = launch_decode_mma(mode, enc, x, w_persist, r, y, M, N, K, stream);
+    } else err = launch_umma_linear(mode, enc, x, w_persist, r, y, M, N, K, d->status, stream);
     return err == cudaSuccess ? DPS_OK : DPS_ERR_CUDA;
 }
 

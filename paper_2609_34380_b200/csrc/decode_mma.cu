@@ -1,0 +1,244 @@
+// Decode linear layer for up to 16 tokens: a register-streaming kernel.
+//
+// Paper: "Scheduler: Dual-Precision Execution" -- fast mode streams the FP8 tensor only, full mode
+// streams the FP8 and the residual tensor and rebuilds the FP16 weights during computation.  With
+// a handful of tokens the layer is a weight stream bound by HBM, so the kernel is built around the
+// stream, not around the arithmetic:
+//   * every warp owns the same 16 weight rows as its CTA and every 8th 64-byte slice of K; each lane
+//     issues 128-bit loads of P (and R) for two rows, several K rounds ahead, so that a CTA keeps
+//     32-64 KB in flight and its eight warps together read 512 contiguous bytes of each row;
+//   * the plane bytes become packed FP16 pairs in registers -- E4M3 fast mode with the hardware
+//     FP8->FP16 conversion (exact, it yields 2^8 times the weight; the factor is taken out at the
+//     store), the other variants with byte permutes -- and those registers ARE the A fragments of
+//     a warp-level m16n8k16 MMA.  The activations are already FP16 pairs, i.e. B fragments.  No
+//     conversion to FP32, no FMA per weight: about one integer instruction per weight;
+//   * the K order inside an MMA is free as long as both operands agree, which is what lets each
+//     lane feed 16 consecutive bytes of one row (four MMAs' worth) without any shuffle;
+//   * partial sums of the eight warps are added in a fixed order through shared memory, so the
+//     result is bit-stable.  CTAs walk the 16-row blocks of the matrix persistently.
+// Tensor memory and TMA buy nothing here (no reuse, nothing to stage); the wide tcgen05 tiles take
+// over once the token count makes the layer a real contraction.
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
+
+#include "bits.cuh"
+#include "dps_internal.h"
+#include "sm100.cuh"
+
+namespace dps {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kRowsPerBlock = 16;
+constexpr int kRoundK = kWarps * 64;  // K covered by the CTA per round: each warp 64 bytes per row
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// D (16x8, FP32) += A (16x16 FP16, row) * B (16x8 FP16, col)
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Four E4M3 bytes -> two packed FP16 pairs holding 2^8 times the weights (exact): one register
+// split and two hardware conversions.
+__device__ __forceinline__ void e4m3x4_to_half2x2(uint32_t w, uint32_t& lo, uint32_t& hi) {
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, l;\n\tcvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
+        : "=r"(lo), "=r"(hi)
+        : "r"(w));
+}
+
+// 16 plane bytes (+ residual bytes) of one row -> 8 packed FP16 pairs, element order preserved.
+// E4M3 fast mode returns 2^8 times the weights; the kernel's kScale undoes it at the store.
+template <int ENC, bool FULL>
+__device__ __forceinline__ void to_half_pairs(const uint4& p, const uint4& r, uint32_t (&h)[8]) {
+    if (ENC == kEncE4M3 && !FULL) {
+        e4m3x4_to_half2x2(p.x, h[0], h[1]);
+        e4m3x4_to_half2x2(p.y, h[2], h[3]);
+        e4m3x4_to_half2x2(p.z, h[4], h[5]);
+        e4m3x4_to_half2x2(p.w, h[6], h[7]);
+    } else {
+        join16<ENC, FULL>(p, r, h);
+    }
+}
+
+// HALF: the CTA owns 8 weight rows instead of 16 (the upper half of every MMA tile is zero).  It
+// doubles the number of CTAs for matrices with few rows; the MMA work wasted is irrelevant here.
+template <int ENC, bool FULL, int NT, int U, bool HALF>
+__global__ void __launch_bounds__(kThreads, 3)
+decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, const uint8_t* __restrict__ Rp,
+                  __half* __restrict__ y, int M, int64_t N, int64_t K) {
+    constexpr float kScale = (ENC == kEncE4M3 && !FULL) ? 0.00390625f : 1.0f;  // 2^-8, exact
+    __shared__ float red[kWarps][kRowsPerBlock][NT * 8 + 1];
+    sm100::grid_launch_dependents();
+    sm100::grid_dependency_wait();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    constexpr int kRows = HALF ? 8 : kRowsPerBlock;
+    const int full_rounds = (int)(K / kRoundK);           // rounds in which every lane is inside K
+    const bool has_tail = (K % kRoundK) != 0;
+    const int kl = warp * 64 + t * 16;                    // this lane's byte offset inside a round
+
+    // activation rows this lane feeds as B fragments (token 8 * n + g of every token group);
+    // lanes without a token read row 0 and have their product discarded at the store
+    const __half* xrow[NT];
+#pragma unroll
+    for (int n = 0; n < NT; ++n) xrow[n] = x + (int64_t)((n * 8 + g < M) ? n * 8 + g : 0) * K + kl;
+
+    {   // one row block per CTA: the hardware block scheduler balances the SMs
+        const int64_t rb = blockIdx.x;
+        // rows past N are clamped for the loads and dropped at the store
+        const int64_t row_lo = rb * kRows + g, row_hi = row_lo + 8;
+        const uint8_t* p_lo = P + (row_lo < N ? row_lo : N - 1) * K + kl;
+        const uint8_t* p_hi = P + (row_hi < N ? row_hi : N - 1) * K + kl;
+        const uint8_t* r_lo = FULL ? Rp + (row_lo < N ? row_lo : N - 1) * K + kl : nullptr;
+        const uint8_t* r_hi = FULL ? Rp + (row_hi < N ? row_hi : N - 1) * K + kl : nullptr;
+        float acc[NT][4];
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[n][c] = 0.f;
+
+        auto multiply = [&](const uint4& wp_lo, const uint4& wp_hi, const uint4& wr_lo, const uint4& wr_hi,
+                            int koff, bool in) {
+            uint32_t a_lo[8], a_hi[8];
+            to_half_pairs<ENC, FULL>(wp_lo, wr_lo, a_lo);
+            if (HALF) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a_hi[i] = 0u;
+            } else {
+                to_half_pairs<ENC, FULL>(wp_hi, wr_hi, a_hi);
+            }
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;
+                if (in) {
+                    b0 = *reinterpret_cast<const uint4*>(xrow[n] + koff);
+                    b1 = *reinterpret_cast<const uint4*>(xrow[n] + koff + 8);
+                }
+                const uint32_t bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                // MMA j takes bytes 4j..4j+3 of the lane's 16: K slots (2t, 2t+1) <- pair 2j and
+                // K slots (2t+8, 2t+9) <- pair 2j+1, for the weights and the activations alike.
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    mma_16816(acc[n], a_lo[2 * j], a_hi[2 * j], a_lo[2 * j + 1], a_hi[2 * j + 1], bb[2 * j],
+                              bb[2 * j + 1]);
+            }
+        };
+
+        int r0 = 0;
+        for (; r0 + U <= full_rounds; r0 += U) {          // U rounds in flight, immediate offsets
+            const int base = r0 * kRoundK;
+            uint4 wp_lo[U], wp_hi[U], wr_lo[U], wr_hi[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                wp_hi[u] = wr_lo[u] = wr_hi[u] = make_uint4(0, 0, 0, 0);
+                wp_lo[u] = ldg_stream(p_lo + base + u * kRoundK);
+                if (!HALF) wp_hi[u] = ldg_stream(p_hi + base + u * kRoundK);
+                if (FULL) {
+                    wr_lo[u] = ldg_stream(r_lo + base + u * kRoundK);
+                    if (!HALF) wr_hi[u] = ldg_stream(r_hi + base + u * kRoundK);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) multiply(wp_lo[u], wp_hi[u], wr_lo[u], wr_hi[u], base + u * kRoundK, true);
+        }
+        for (; r0 < full_rounds + (has_tail ? 1 : 0); ++r0) {   // leftover rounds and the ragged end of K
+            const int base = r0 * kRoundK;
+            if ((int64_t)base + warp * 64 >= K) continue;       // warp-uniform: the MMA needs the whole warp
+            const bool in = (int64_t)base + kl < K;
+            uint4 wp_lo = make_uint4(0, 0, 0, 0), wp_hi = wp_lo, wr_lo = wp_lo, wr_hi = wp_lo;
+            if (in) {
+                wp_lo = ldg_stream(p_lo + base);
+                if (!HALF) wp_hi = ldg_stream(p_hi + base);
+                if (FULL) {
+                    wr_lo = ldg_stream(r_lo + base);
+                    if (!HALF) wr_hi = ldg_stream(r_hi + base);
+                }
+            }
+            multiply(wp_lo, wp_hi, wr_lo, wr_hi, base, in);
+        }
+        // accumulator fragment: c0,c1 = (row g, tokens 2t, 2t+1), c2,c3 = (row g+8, same tokens)
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+            red[warp][g][n * 8 + 2 * t] = acc[n][0];
+            red[warp][g][n * 8 + 2 * t + 1] = acc[n][1];
+            if (!HALF) {
+                red[warp][g + 8][n * 8 + 2 * t] = acc[n][2];
+                red[warp][g + 8][n * 8 + 2 * t + 1] = acc[n][3];
+            }
+        }
+        __syncthreads();
+        for (int o = threadIdx.x; o < kRows * NT * 8; o += kThreads) {
+            const int tok = o / kRows, row = o % kRows;
+            const int64_t n_out = rb * kRows + row;
+            if (tok < M && n_out < N) {
+                float s = 0.f;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) s += red[w][row][tok];
+                y[(int64_t)tok * N + n_out] = __float2half_rn(s * kScale);
+            }
+        }
+        __syncthreads();
+    }
+}
+
+template <int ENC, bool FULL, int NT, int U, bool HALF>
+cudaError_t launch_one(const __half* x, const uint8_t* p, const uint8_t* r, __half* y, int M, int64_t N, int64_t K,
+                       cudaStream_t stream) {
+    constexpr int kRows = HALF ? 8 : kRowsPerBlock;
+    const int64_t grid = (N + kRows - 1) / kRows;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_mma_kernel<ENC, FULL, NT, U, HALF>, x, p, r, y, M, N, K);
+    count_launch();
+    return e;
+}
+
+template <int ENC, bool FULL>
+cudaError_t launch_enc(const __half* x, const uint8_t* p, const uint8_t* r, __half* y, int M, int64_t N, int64_t K,
+                       cudaStream_t stream) {
+    // Rounds in flight per lane: 128 bytes either way (fast mode reads one plane per round).
+    // Half-height blocks were measured slower for every Llama-7B shape (the kernel is bound by
+    // instruction issue, and they double the MMA and activation-load instructions per weight), so
+    // they stay off.
+    constexpr int U = FULL ? 2 : 4;
+    if (M <= 8) return launch_one<ENC, FULL, 1, U, false>(x, p, r, y, M, N, K, stream);
+    return launch_one<ENC, FULL, 2, U, false>(x, p, r, y, M, N, K, stream);
+}
+
+}  // namespace
+
+cudaError_t launch_decode_mma(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
+                              int64_t M, int64_t N, int64_t K, cudaStream_t stream) {
+    const __half* xh = static_cast<const __half*>(x);
+    __half* yh = static_cast<__half*>(y);
+    const bool full = mode == DPS_MODE_FULL;
+    if (enc == kEncE4M3)
+        return full ? launch_enc<kEncE4M3, true>(xh, p, r, yh, (int)M, N, K, stream)
+                    : launch_enc<kEncE4M3, false>(xh, p, r, yh, (int)M, N, K, stream);
+    return full ? launch_enc<kEncE5M2, true>(xh, p, r, yh, (int)M, N, K, stream)
+                : launch_enc<kEncE5M2, false>(xh, p, r, yh, (int)M, N, K, stream);
+}
+
+}  // namespace dps

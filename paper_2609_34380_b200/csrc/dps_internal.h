@@ -21,6 +21,10 @@ cudaError_t launch_reconstruct(const uint8_t* p, const uint8_t* r, uint16_t* w, 
 cudaError_t launch_gemv(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
                         int64_t M, int64_t N, int64_t K, cudaStream_t stream);
 
+// Dense linear for M <= 16: register-streaming kernel with warp-level MMAs.
+cudaError_t launch_decode_mma(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
+                              int64_t M, int64_t N, int64_t K, cudaStream_t stream);
+
 // Dense linear, tensor-core path (tcgen05 + TMEM).  `status` receives DPS_ERR_CUDA if a bounded
 // wait inside the kernel ever gives up.
 cudaError_t launch_umma_linear(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,

@@ -1,6 +1,7 @@
 // Dense linear layer on the CUDA-core GEMV path (see gemv.cuh for the design).
 #include "dps_internal.h"
 #include "gemv.cuh"
+#include "sm100.cuh"
 
 namespace dps {
 
@@ -11,6 +12,8 @@ __global__ void __launch_bounds__(kGemvThreads, 2)
 gemv_dense_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, const uint8_t* __restrict__ Rp,
                   __half* __restrict__ y, int m_count, int64_t N, int64_t K, int rows_per_cta, int red_stride) {
     extern __shared__ float red[];
+    sm100::grid_launch_dependents();  // let the next kernel's CTAs take the slots this grid frees
+    sm100::grid_dependency_wait();    // activations (and possibly planes) come from the preceding kernel
     const int64_t row_begin = (int64_t)blockIdx.x * rows_per_cta;
     const int64_t row_end = (row_begin + rows_per_cta < N) ? row_begin + rows_per_cta : N;
     if (row_begin >= row_end) return;
@@ -36,10 +39,20 @@ cudaError_t launch_one(const __half* x, const uint8_t* p, const uint8_t* r, __ha
     const int64_t grid = (N + rows - 1) / rows;
     const int red_stride = (int)((rows + kGemvRows - 1) / kGemvRows) * kGemvRows * MT;
     const size_t smem = (size_t)kGemvWarps * red_stride * sizeof(float);
-    gemv_dense_kernel<ENC, FULL, MT><<<(unsigned)grid, kGemvThreads, smem, stream>>>(x, p, r, y, m_count, N, K,
-                                                                                     (int)rows, red_stride);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kGemvThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemv_dense_kernel<ENC, FULL, MT>, x, p, r, y, m_count, N, K, (int)rows,
+                                       red_stride);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 template <int ENC, bool FULL>

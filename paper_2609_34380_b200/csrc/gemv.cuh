@@ -18,7 +18,9 @@ namespace dps {
 
 constexpr int kGemvThreads = 256;
 constexpr int kGemvWarps = kGemvThreads / 32;
-constexpr int kGemvRows = 8;                      // weight rows in flight per thread
+constexpr int kGemvRows = 8;                      // weight rows reduced together (one butterfly)
+constexpr int kGemvBatch = 2;                     // row groups whose loads are issued together when only
+                                                  // one plane is read, so both modes keep 256 B per thread in flight
 constexpr int kGemvKPass = kGemvThreads * 16;     // K covered by one pass of the CTA
 
 __device__ __forceinline__ uint4 ldg_stream16(const void* p) {
@@ -86,39 +88,48 @@ __device__ __forceinline__ void gemv_rows(const __half* const (&xrow)[MT], __hal
                 xf[t][2 * j + 1] = f.y;
             }
         }
-        for (int b = 0; b < nblocks; ++b) {
-            uint4 pw[kGemvRows], rw[kGemvRows];
+        constexpr int kBatch = FULL ? 1 : kGemvBatch;
+        for (int b0 = 0; b0 < nblocks; b0 += kBatch) {
+            uint4 pw[kBatch][kGemvRows], rw[kBatch][kGemvRows];
 #pragma unroll
-            for (int i = 0; i < kGemvRows; ++i) {
-                const int64_t row = row_begin + (int64_t)b * kGemvRows + i;
-                pw[i] = make_uint4(0, 0, 0, 0);
-                rw[i] = make_uint4(0, 0, 0, 0);
-                if (active && row < row_end) {
-                    pw[i] = ldg_stream16(P + row * K + k);
-                    if (FULL) rw[i] = ldg_stream16(Rp + row * K + k);
-                }
-            }
-            float acc[V];
+            for (int u = 0; u < kBatch; ++u) {
 #pragma unroll
-            for (int v = 0; v < V; ++v) acc[v] = 0.f;
-#pragma unroll
-            for (int i = 0; i < kGemvRows; ++i) {
-                uint32_t h[8];
-                join16<ENC, FULL>(pw[i], rw[i], h);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float2 w = h2f2(h[j]);
-#pragma unroll
-                    for (int t = 0; t < MT; ++t) {
-                        acc[i * MT + t] = fmaf(w.x, xf[t][2 * j], acc[i * MT + t]);
-                        acc[i * MT + t] = fmaf(w.y, xf[t][2 * j + 1], acc[i * MT + t]);
+                for (int i = 0; i < kGemvRows; ++i) {
+                    const int64_t row = row_begin + (int64_t)(b0 + u) * kGemvRows + i;
+                    pw[u][i] = make_uint4(0, 0, 0, 0);
+                    rw[u][i] = make_uint4(0, 0, 0, 0);
+                    if (active && row < row_end) {
+                        pw[u][i] = ldg_stream16(P + row * K + k);
+                        if (FULL) rw[u][i] = ldg_stream16(Rp + row * K + k);
                     }
                 }
             }
-            const float s = butterfly_sum<V>(acc, lane);
-            if ((lane & (kGroup - 1)) == 0) {
-                float* slot = red + warp * red_stride + b * V + (lane / kGroup);
-                *slot = (k0 == 0) ? s : (*slot + s);
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int b = b0 + u;
+                if (b >= nblocks) break;
+                float acc[V];
+#pragma unroll
+                for (int v = 0; v < V; ++v) acc[v] = 0.f;
+#pragma unroll
+                for (int i = 0; i < kGemvRows; ++i) {
+                    uint32_t h[8];
+                    join16<ENC, FULL>(pw[u][i], rw[u][i], h);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float2 w = h2f2(h[j]);
+#pragma unroll
+                        for (int t = 0; t < MT; ++t) {
+                            acc[i * MT + t] = fmaf(w.x, xf[t][2 * j], acc[i * MT + t]);
+                            acc[i * MT + t] = fmaf(w.y, xf[t][2 * j + 1], acc[i * MT + t]);
+                        }
+                    }
+                }
+                const float s = butterfly_sum<V>(acc, lane);
+                if ((lane & (kGroup - 1)) == 0) {
+                    float* slot = red + warp * red_stride + b * V + (lane / kGroup);
+                    *slot = (k0 == 0) ? s : (*slot + s);
+                }
             }
         }
     }

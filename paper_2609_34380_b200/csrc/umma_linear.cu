@@ -256,6 +256,18 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         // Stages are filled two at a time when the ring is deep enough: the two boxes cover 256
         // adjacent bytes of every weight row, which DRAM serves noticeably better than 128.
         const bool pair = (num_stages >= 6) && (num_stages % 2 == 0);
+        // While the preceding kernel drains, pull this CTA's first plane tiles into L2.  L2 is the
+        // point of coherence, so this is safe even if that kernel is still writing the planes; the
+        // loads proper are issued only after the dependency wait.
+        if (!GROUPED && elect_one()) {
+            const int ahead = num_kb < 2 * num_stages ? num_kb : 2 * num_stages;
+            for (int i = 0; i < ahead; ++i) {
+                const int k = (rank + i * split) * kBlockK;
+                tma_prefetch_l2_2d(&map_p, k, plane_row0);
+                if (FULL) tma_prefetch_l2_2d(&map_r, k, plane_row0);
+            }
+        }
+        __syncwarp();
         grid_dependency_wait();  // everything read from global memory may come from the preceding kernel
         for (int i = 0; i < num_kb && ok; ++i) {
             const int s = i % num_stages;
