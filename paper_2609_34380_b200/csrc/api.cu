@@ -170,7 +170,7 @@ dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w
     if (path == 1) err = launch_gemv(mode, enc, x, w_persist, r, y, M, N, K, stream);
     else if (path == 2) err = launch_umma_linear(mode, enc, x, w_persist, r, y, M, N, K, d->status, stream);
     else if (path == 3 || M <= 16) {
-        if (M > 16) return DPS_ERR_UNSUPPORTED;
+        if (M > 32) return DPS_ERR_UNSUPPORTED;
         err = launch_decode_mma(mode, enc, x, w_persist, r, y, M, N, K, stream);
     } else err = launch_umma_linear(mode, enc, x, w_persist, r, y, M, N, K, d->status, stream);
     return err == cudaSuccess ? DPS_OK : DPS_ERR_CUDA;

@@ -224,7 +224,8 @@ cudaError_t launch_enc(const __half* x, const uint8_t* p, const uint8_t* r, __ha
     // they stay off.
     constexpr int U = FULL ? 2 : 4;
     if (M <= 8) return launch_one<ENC, FULL, 1, U, false>(x, p, r, y, M, N, K, stream);
-    return launch_one<ENC, FULL, 2, U, false>(x, p, r, y, M, N, K, stream);
+    if (M <= 16) return launch_one<ENC, FULL, 2, U, false>(x, p, r, y, M, N, K, stream);
+    return launch_one<ENC, FULL, 4, U, false>(x, p, r, y, M, N, K, stream);
 }
 
 }  // namespace

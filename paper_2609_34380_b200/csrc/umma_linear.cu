@@ -195,8 +195,23 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_stages = prm.num_stages;
-    const int n0 = blockIdx.x * kTileRows;
-    int m0 = blockIdx.y * TN;        // first token (dense) / first sorted row (grouped) of the tile
+    // Tile order (dense launches with several token tiles): CTAs are handed out x-fastest, so walk
+    // groups of 8 row tiles x all token tiles.  The CTAs running at any moment then share 8 row
+    // tiles of planes and a few dozen activation tiles, which stay in L2, instead of sweeping
+    // the whole weight matrix once per token tile (measured: 1.04 GB of DRAM reads for a
+    // 100 MB full-mode QKV layer at 2048 tokens before this, because P + R no longer fit in L2).
+    int row_tile = blockIdx.x, tok_tile = blockIdx.y;
+    if (!GROUPED && gridDim.y > 1) {
+        constexpr int kRowGroup = 8;
+        const int lin = blockIdx.x + gridDim.x * blockIdx.y;
+        const int per_group = kRowGroup * gridDim.y;
+        const int group = lin / per_group, within = lin % per_group;
+        const int rows_here = min(kRowGroup, (int)gridDim.x - group * kRowGroup);
+        row_tile = group * kRowGroup + within % rows_here;
+        tok_tile = within / rows_here;
+    }
+    const int n0 = row_tile * kTileRows;
+    int m0 = tok_tile * TN;          // first token (dense) / first sorted row (grouped) of the tile
     int tile_tokens = TN;            // valid token columns of the tile (grouped)
     int plane_row0 = n0;             // first plane row of the tile in the [E * N][K] view
     bool e5m2 = (ENC == kEncE5M2);
@@ -590,7 +605,16 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
     if (M <= 16) return launch_tn<ENC, FULL, 16>(x, p, r, y, M, N, K, status, stream);
     if (M <= 32) return launch_tn<ENC, FULL, 32>(x, p, r, y, M, N, K, status, stream);
     if (M <= 64) return launch_tn<ENC, FULL, 64>(x, p, r, y, M, N, K, status, stream);
-    if (M <= 128 || M > 256) return launch_tn<ENC, FULL, 128>(x, p, r, y, M, N, K, status, stream);
+    // Prefill: in full mode the zip warps (two planes to read, more bit work) are the bottleneck,
+    // and a 256-token tile halves their work per FLOP (one CTA per SM, each rebuilt weight block
+    // feeds twice the columns); in fast mode two co-resident 128-token CTAs with deeper rings win.
+    // DPS_FORCE_TN=128|256 overrides (tuning knob).
+    static const int tn_forced = [] {
+        const char* e = getenv("DPS_FORCE_TN");
+        return e ? atoi(e) : 0;
+    }();
+    const bool wide = tn_forced ? tn_forced == 256 : (FULL ? M > 128 : (M > 128 && M <= 256));
+    if (!wide) return launch_tn<ENC, FULL, 128>(x, p, r, y, M, N, K, status, stream);
     return launch_tn<ENC, FULL, 256>(x, p, r, y, M, N, K, status, stream);
 }
 
