@@ -60,6 +60,32 @@ __device__ __forceinline__ void split4(uint32_t a, uint32_t b, uint32_t& p4, uin
     r4 = __byte_perm(a, b, 0x6420);  // low bytes
 }
 
+// Four E4M3 bytes -> two packed FP16 pairs holding 2^8 times the fast-mode weights: one register
+// split and two hardware conversions.  Exact for every legal byte (the E4M3 value of the byte is
+// 2^8 times the weight, subnormals included; the code 0x7F/0xFF never occurs in a legal plane),
+// so a kernel may multiply with these and scale its result by 2^-8 at the end.
+__device__ __forceinline__ void e4m3x4_to_half2x2_scaled(uint32_t w, uint32_t& lo, uint32_t& hi) {
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, l;\n\tcvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
+        : "=r"(lo), "=r"(hi)
+        : "r"(w));
+}
+
+// 16 persistent bytes -> 16 FP16 words for FAST mode, E4M3 through the hardware conversion
+// (result scaled by 2^8, see above), E5M2 by byte permutes (unscaled).
+template <int ENC>
+__device__ __forceinline__ void fast16(const uint4& p, uint32_t (&h)[8]) {
+    if (ENC == kEncE4M3) {
+        e4m3x4_to_half2x2_scaled(p.x, h[0], h[1]);
+        e4m3x4_to_half2x2_scaled(p.y, h[2], h[3]);
+        e4m3x4_to_half2x2_scaled(p.z, h[4], h[5]);
+        e4m3x4_to_half2x2_scaled(p.w, h[6], h[7]);
+    } else {
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+        join16<ENC, false>(p, zero, h);
+    }
+}
+
 __device__ __forceinline__ float2 h2f2(uint32_t h2) {
     return __half22float2(*reinterpret_cast<const __half2*>(&h2));
 }

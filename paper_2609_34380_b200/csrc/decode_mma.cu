@@ -51,27 +51,12 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Four E4M3 bytes -> two packed FP16 pairs holding 2^8 times the weights (exact): one register
-// split and two hardware conversions.
-__device__ __forceinline__ void e4m3x4_to_half2x2(uint32_t w, uint32_t& lo, uint32_t& hi) {
-    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\t"
-        "cvt.rn.f16x2.e4m3x2 %0, l;\n\tcvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
-        : "=r"(lo), "=r"(hi)
-        : "r"(w));
-}
-
 // 16 plane bytes (+ residual bytes) of one row -> 8 packed FP16 pairs, element order preserved.
 // E4M3 fast mode returns 2^8 times the weights; the kernel's kScale undoes it at the store.
 template <int ENC, bool FULL>
 __device__ __forceinline__ void to_half_pairs(const uint4& p, const uint4& r, uint32_t (&h)[8]) {
-    if (ENC == kEncE4M3 && !FULL) {
-        e4m3x4_to_half2x2(p.x, h[0], h[1]);
-        e4m3x4_to_half2x2(p.y, h[2], h[3]);
-        e4m3x4_to_half2x2(p.z, h[4], h[5]);
-        e4m3x4_to_half2x2(p.w, h[6], h[7]);
-    } else {
-        join16<ENC, FULL>(p, r, h);
-    }
+    if (!FULL) fast16<ENC>(p, h);
+    else join16<ENC, FULL>(p, r, h);
 }
 
 // HALF: the CTA owns 8 weight rows instead of 16 (the upper half of every MMA tile is zero).  It

@@ -40,7 +40,8 @@ constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
 constexpr int kBlockK = 128;     // K elements per pipeline stage: 128-byte plane rows, the widest swizzled TMA box
 constexpr int kXAtoms = kBlockK / 64;  // the x tile is stored as 64-element (128-byte) swizzle atoms
 constexpr int kACols = kBlockK / 2;    // TMEM columns of one A stage (two FP16 per column)
-constexpr int kAStages = 2;      // A ring in tensor memory
+constexpr int kAStages = 2;      // A ring in tensor memory when the stage ring has an even depth
+constexpr int kMaxAStages = 3;   // with a 3-deep stage ring every stage has its own A slot
 constexpr int kZipGroups = 2;    // groups of 4 zip warps; group g takes K blocks g, g + G, ...
 constexpr int kThreads = 64 + kZipGroups * 128;
 constexpr int kPlaneStageBytes = kTileRows * kBlockK;  // 16 KB per plane per stage
@@ -51,8 +52,11 @@ static_assert(kAStages % kZipGroups == 0, "each A stage must belong to one zip g
 __host__ __device__ constexpr int stage_bytes(bool full, int tn) {
     return kPlaneStageBytes * (full ? 2 : 1) + tn * kBlockK * 2;
 }
+// Columns to allocate: accumulator + A ring.  Tiles of up to 64 tokens leave room for three A
+// slots inside 256 columns (two CTAs per SM); wider tiles keep two.
+__host__ __device__ constexpr int a_slots_max(int tn) { return tn <= 64 ? kMaxAStages : kAStages; }
 __host__ __device__ constexpr int tmem_cols(int tn) {
-    int need = tn + kAStages * kACols;
+    int need = tn + a_slots_max(tn) * kACols;
     int c = 32;
     while (c < need) c <<= 1;
     return c;
@@ -106,6 +110,7 @@ struct UmmaParams {
 // What a zip warp needs to know about its CTA's pipeline.
 struct ZipCtx {
     int group, warp, lane, row, num_kb, num_stages, stage_bytes;
+    bool slot_per_stage;  // 3-deep ring: A slot = stage, owner group = stage % groups
     uint32_t smem_base, tmem_a, lane_base, sw;
     uint64_t *bar_full, *bar_empty, *bar_a_full, *bar_a_empty;
 };
@@ -116,12 +121,22 @@ struct ZipCtx {
 template <int ENC, bool FULL>
 __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
     bool ok = true;
-    for (int i = z.group; i < z.num_kb && ok; i += kZipGroups) {
-        const int s = i % z.num_stages, a = i % kAStages;
+    // Ring positions are advanced incrementally (no division in the loop).  Every stage and every A
+    // slot always belongs to the same zip group, so that each waiter sees every phase of the barriers
+    // it waits on.  Even ring: blocks alternate between the groups and between two A slots.
+    // 3-deep ring: slot = stage, group = stage % groups.
+    int s = 0;
+    uint32_t s_parity = 0, pair_parity = 0;   // phase parity of stage s; parity of (i / 2)
+    for (int i = 0; i < z.num_kb && ok;
+         ++i, pair_parity ^= (uint32_t)(i & 1) ^ 1u, s = (s + 1 == z.num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
+        const int a = z.slot_per_stage ? s : (i & 1);
+        const int owner = z.slot_per_stage ? (s & 1) : (i & 1);
+        if (owner != z.group) continue;
+        const uint32_t a_parity = z.slot_per_stage ? s_parity : pair_parity;
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(4, i);
-        ok = mbar_wait(smem_u32(&z.bar_full[s]), (uint32_t)(i / z.num_stages) & 1u);
+        ok = mbar_wait(smem_u32(&z.bar_full[s]), s_parity);
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(5, i);
-        if (ok) ok = mbar_wait(smem_u32(&z.bar_a_empty[a]), ((uint32_t)(i / kAStages) & 1u) ^ 1u);
+        if (ok) ok = mbar_wait(smem_u32(&z.bar_a_empty[a]), a_parity ^ 1u);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(6, i);
@@ -140,7 +155,8 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
                              : "=r"(rv.x), "=r"(rv.y), "=r"(rv.z), "=r"(rv.w)
                              : "r"(prow + kPlaneStageBytes + off));
             uint32_t h8[8];
-            join16<ENC, FULL>(pv, rv, h8);
+            if (FULL) join16<ENC, FULL>(pv, rv, h8);
+            else fast16<ENC>(pv, h8);   // E4M3: 2^8 times the weights, undone in the epilogue
 #pragma unroll
             for (int j = 0; j < 8; ++j) h[c * 8 + j] = h8[j];
         }
@@ -177,8 +193,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[kMaxStages];
     __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
-    __shared__ __align__(8) uint64_t bar_a_full[kAStages];
-    __shared__ __align__(8) uint64_t bar_a_empty[kAStages];
+    __shared__ __align__(8) uint64_t bar_a_full[kMaxAStages];
+    __shared__ __align__(8) uint64_t bar_a_empty[kMaxAStages];
     __shared__ __align__(8) uint64_t bar_d_full;
     __shared__ uint32_t tmem_base_slot;
 
@@ -195,6 +211,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_stages = prm.num_stages;
+    const bool slot_per_stage = (num_stages % kZipGroups) != 0;   // only the 3-deep ring
     // Tile order (dense launches with several token tiles): CTAs are handed out x-fastest, so walk
     // groups of 8 row tiles x all token tiles.  The CTAs running at any moment then share 8 row
     // tiles of planes and a few dozen activation tiles, which stay in L2, instead of sweeping
@@ -236,7 +253,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             mbar_init(smem_u32(&bar_full[s]), 1);
             mbar_init(smem_u32(&bar_empty[s]), 5);  // 4 zip warps + 1 tcgen05.commit
         }
-        for (int a = 0; a < kAStages; ++a) {
+        for (int a = 0; a < kMaxAStages; ++a) {
             mbar_init(smem_u32(&bar_a_full[a]), 4);
             mbar_init(smem_u32(&bar_a_empty[a]), 1);
         }
@@ -284,14 +301,14 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         }
         __syncwarp();
         grid_dependency_wait();  // everything read from global memory may come from the preceding kernel
-        for (int i = 0; i < num_kb && ok; ++i) {
-            const int s = i % num_stages;
-            const uint32_t ph = (uint32_t)(i / num_stages) & 1u;
+        int s = 0;
+        uint32_t ph = 0;
+        for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
             if (!pair || (i & 1) == 0) {
                 ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);
-                if (ok && pair && i + 1 < num_kb)
-                    ok = mbar_wait(smem_u32(&bar_empty[(i + 1) % num_stages]),
-                                   ((uint32_t)((i + 1) / num_stages) & 1u) ^ 1u);
+                if (ok && pair && i + 1 < num_kb) {     // pairs never wrap: the ring depth is even
+                    ok = mbar_wait(smem_u32(&bar_empty[s + 1]), ph ^ 1u);
+                }
             }
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
@@ -311,11 +328,15 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (whole warp converged, one elected lane issues) ----------------
-        for (int i = 0; i < num_kb && ok; ++i) {
-            const int s = i % num_stages, a = i % kAStages;
-            ok = mbar_wait(smem_u32(&bar_full[s]), (uint32_t)(i / num_stages) & 1u);
+        int s = 0;
+        uint32_t s_parity = 0, pair_parity = 0;
+        for (int i = 0; i < num_kb && ok;
+             ++i, pair_parity ^= (uint32_t)(i & 1) ^ 1u, s = (s + 1 == num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
+            const int a = slot_per_stage ? s : (i & 1);
+            // The zip warps waited for this stage's TMA loads before they arrived on a_full, so the
+            // activation tile of the stage is complete and visible once a_full is: one wait, not two.
             DPS_STAMP(1, i);
-            if (ok) ok = mbar_wait(smem_u32(&bar_a_full[a]), (uint32_t)(i / kAStages) & 1u);
+            ok = mbar_wait(smem_u32(&bar_a_full[a]), slot_per_stage ? s_parity : pair_parity);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             DPS_STAMP(2, i);
@@ -346,6 +367,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         ZipCtx zc;
         zc.group = group; zc.warp = warp; zc.lane = lane; zc.row = row;
         zc.num_kb = num_kb; zc.num_stages = num_stages; zc.stage_bytes = kStage;
+        zc.slot_per_stage = slot_per_stage;
         zc.smem_base = smem_base; zc.tmem_a = tmem_a; zc.lane_base = lane_base;
         zc.sw = (uint32_t)(row & 7);  // 128-byte swizzle: 16-byte chunk index ^= row % 8
         zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
@@ -357,6 +379,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         }
         // epilogue (first zip group): D[row][token] -> y[token][n0 + row], or -> red for split K
         if (group == 0) {
+            // E4M3 fast mode multiplied with 2^8 times the weights (hardware FP8 conversion)
+            const float out_scale = (!FULL && !e5m2) ? 0.00390625f : 1.0f;
             if (ok) ok = mbar_wait(smem_u32(&bar_d_full), 0u);
             ok = __all_sync(0xFFFFFFFFu, ok);
             DPS_CTA_STAMP(2);
@@ -373,11 +397,12 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                         for (int j = 0; j < 16; ++j) {
                             const int c = c0 + j, owner = c % split, slot = c / split;
                             const uint32_t local = mail_addr + (uint32_t)(((rank * slots + slot) * kTileRows + row) * 4);
-                            st_cluster_f32(map_to_cta(local, (uint32_t)owner), __uint_as_float(v[j]));
+                            st_cluster_f32(map_to_cta(local, (uint32_t)owner), __uint_as_float(v[j]) * out_scale);
                         }
                     } else if (split > 1) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) red[(c0 + j) * kTileRows + row] = __uint_as_float(v[j]);
+                        for (int j = 0; j < 16; ++j)
+                            red[(c0 + j) * kTileRows + row] = __uint_as_float(v[j]) * out_scale;
                     } else if (n < prm.N) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
@@ -387,7 +412,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                                 valid = (c0 + j) < tile_tokens;
                                 if (valid) m = gp.sorted_rows[m];
                             }
-                            if (valid) prm.y[(int64_t)m * prm.N + n] = __float2half_rn(__uint_as_float(v[j]));
+                            if (valid)
+                                prm.y[(int64_t)m * prm.N + n] = __float2half_rn(__uint_as_float(v[j]) * out_scale);
                         }
                     }
                 }
@@ -498,13 +524,17 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     constexpr int kStage = stage_bytes(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(TN) <= 256 ? 2 : 1;
     constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
-    constexpr int kMailBytes = TN <= 64 ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox
-    int stages = (kSmemTotal - kMailBytes) / kStage;
-    if (stages > 8) stages = 8;
-    if (stages < 2) stages = 2;
-    stages -= stages % kZipGroups;  // a stage always belongs to the same zip group, so that every
-                                    // waiter sees every phase of the barriers it waits on
-    const size_t smem = (size_t)stages * kStage + kMailBytes + 1024;
+    constexpr int kMailMax = TN <= 64 ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox, worst case
+    // Ring depth for a given mailbox size: even, or exactly 3 (every stage then owns an A slot,
+    // which needs a tile of at most 64 tokens).
+    auto ring_depth = [&](int mail_bytes) {
+        int d = (kSmemTotal - mail_bytes) / kStage;
+        if (d > 8) d = 8;
+        if (d < 2) d = 2;
+        if (d % kZipGroups != 0 && !(d == 3 && a_slots_max(TN) >= 3)) d -= d % kZipGroups;
+        return d;
+    };
+    const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kMailMax + 1024;
     auto kernel = umma_linear_kernel<ENC, FULL, TN, false>;
     static int capacity[kMaxSplit + 1] = {0};  // per instantiation; filled on first use
     static bool configured = false;
@@ -520,7 +550,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
             cudaLaunchConfig_t q = {};
             q.gridDim = dim3(1, 1, (unsigned)s);
             q.blockDim = dim3(kThreads, 1, 1);
-            q.dynamicSmemBytes = smem;
+            q.dynamicSmemBytes = smem_query;
             cudaLaunchAttribute qa[1];
             qa[0].id = cudaLaunchAttributeClusterDimension;
             qa[0].val.clusterDim.x = 1;
@@ -562,7 +592,12 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     if (split <= 0) split = choose_split(row_tiles * tok_tiles, total_kb, capacity);
     if (split > total_kb) split = total_kb;
     if (split > kMaxSplit) split = kMaxSplit;
-    if (kMailBytes == 0 && (size_t)stages * kStage < (size_t)TN * kTileRows * 4) split = 1;  // pull mode overlays the ring
+    // the mailbox exists only when K is split, and then has its exact size
+    const int slots = split > 1 ? (TN + split - 1) / split : 0;
+    const int mail_bytes = (split > 1 && kMailMax > 0) ? split * slots * kTileRows * 4 : 0;
+    const int stages = ring_depth(mail_bytes);
+    const size_t smem = (size_t)stages * kStage + mail_bytes + 1024;
+    if (kMailMax == 0 && (size_t)stages * kStage < (size_t)TN * kTileRows * 4) split = 1;  // pull mode overlays the ring
     if (getenv("DPS_DEBUG"))
         fprintf(stderr, "[dps] umma TN=%d full=%d N=%lld K=%lld M=%lld stages=%d split=%d capacity=%d,%d,%d,%d,%d,%d,%d,%d\n",
                 TN, (int)FULL, (long long)N, (long long)K, (long long)M, stages, split, capacity[1], capacity[2],
