@@ -24,19 +24,19 @@ __device__ __forceinline__ uint32_t e4m3_zipped_to_half2(uint32_t z) {
 template <int ENC, bool FULL>
 __device__ __forceinline__ void join4(uint32_t p4, uint32_t r4, uint32_t& lo, uint32_t& hi) {
     if (!FULL) r4 = 0u;
-    uint32_t zl = __byte_perm(r4, p4, 0x5140);  // r0 p0 r1 p1 (low byte first)
-    uint32_t zh = __byte_perm(r4, p4, 0x7362);  // r2 p2 r3 p3
     if (ENC == kEncE4M3) {
-        if (FULL) {
-            zl = e4m3_zipped_to_half2(zl);
-            zh = e4m3_zipped_to_half2(zh);
-        } else {  // residual is zero: only the sign and the seven kept bits move
-            zl = (zl & 0x80008000u) | ((zl >> 1) & 0x3F803F80u);
-            zh = (zh & 0x80008000u) | ((zh >> 1) & 0x3F803F80u);
-        }
+        // Do the E4M3 bit moves on four bytes at a time, BEFORE zipping (7 operations per four
+        // weights instead of 10):
+        //   high byte of the FP16 word = s 0 e3 e2 e1 e0 m9 m8  = (p & 0x80) | ((p & 0x7F) >> 1)
+        //   low  byte of the FP16 word = m7 m6 .. m0            = ((p & 1) << 7) | (r & 0x7F)
+        const uint32_t hi_bytes = (p4 & 0x80808080u) | ((p4 >> 1) & 0x3F3F3F3Fu);
+        const uint32_t lo_bytes = ((p4 << 7) & 0x80808080u) | (r4 & 0x7F7F7F7Fu);
+        lo = __byte_perm(lo_bytes, hi_bytes, 0x5140);
+        hi = __byte_perm(lo_bytes, hi_bytes, 0x7362);
+    } else {
+        lo = __byte_perm(r4, p4, 0x5140);  // r0 p0 r1 p1 (low byte first)
+        hi = __byte_perm(r4, p4, 0x7362);  // r2 p2 r3 p3
     }
-    lo = zl;
-    hi = zh;
 }
 
 // 16 plane bytes (+16 residual bytes) -> 16 FP16 words as 8 packed registers.

@@ -291,8 +291,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         // While the preceding kernel drains, pull this CTA's first plane tiles into L2.  L2 is the
         // point of coherence, so this is safe even if that kernel is still writing the planes; the
         // loads proper are issued only after the dependency wait.
-        if (!GROUPED && elect_one()) {
-            const int ahead = num_kb < 2 * num_stages ? num_kb : 2 * num_stages;
+        // (A rolling L2 prefetch further ahead during the main loop was measured slower.)
+        const int l2_ahead = 2 * num_stages;
+        if (elect_one()) {
+            const int ahead = num_kb < l2_ahead ? num_kb : l2_ahead;
             for (int i = 0; i < ahead; ++i) {
                 const int k = (rank + i * split) * kBlockK;
                 tma_prefetch_l2_2d(&map_p, k, plane_row0);
@@ -527,8 +529,16 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     constexpr int kMailMax = TN <= 64 ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox, worst case
     // Ring depth for a given mailbox size: even, or exactly 3 (every stage then owns an A slot,
     // which needs a tile of at most 64 tokens).
+    static const int deep_forced = [] {
+        const char* e = getenv("DPS_FORCE_DEEP");
+        return e ? atoi(e) : -1;
+    }();
+    const int64_t tiles_total = ((N + kTileRows - 1) / kTileRows) * ((M + TN - 1) / TN);
+    // One CTA per SM with a ring twice as deep when the tiles cannot fill two CTA slots per SM anyway.
+    const bool deep = deep_forced >= 0 ? deep_forced != 0 : false;
+    const int smem_total = (deep || kCtasPerSm == 1) ? 216 * 1024 : kSmemTotal;
     auto ring_depth = [&](int mail_bytes) {
-        int d = (kSmemTotal - mail_bytes) / kStage;
+        int d = (smem_total - mail_bytes) / kStage;
         if (d > 8) d = 8;
         if (d < 2) d = 2;
         if (d % kZipGroups != 0 && !(d == 3 && a_slots_max(TN) >= 3)) d -= d % kZipGroups;
@@ -590,6 +600,8 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     const int total_kb = (int)((K + kBlockK - 1) / kBlockK);
     int split = forced_split();
     if (split <= 0) split = choose_split(row_tiles * tok_tiles, total_kb, capacity);
+    if (deep) split = 1;
+    (void)tiles_total;
     if (split > total_kb) split = total_kb;
     if (split > kMaxSplit) split = kMaxSplit;
     // the mailbox exists only when K is split, and then has its exact size
