@@ -21,6 +21,8 @@
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
 
+#include <cstdlib>
+
 #include "bits.cuh"
 #include "dps_internal.h"
 #include "sm100.cuh"
@@ -62,7 +64,7 @@ __device__ __forceinline__ void to_half_pairs(const uint4& p, const uint4& r, ui
 // HALF: the CTA owns 8 weight rows instead of 16 (the upper half of every MMA tile is zero).  It
 // doubles the number of CTAs for matrices with few rows; the MMA work wasted is irrelevant here.
 template <int ENC, bool FULL, int NT, int U, bool HALF>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, (U * (FULL ? 2 : 1) >= 8 ? 2 : 3))
 decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, const uint8_t* __restrict__ Rp,
                   __half* __restrict__ y, int M, int64_t N, int64_t K) {
     constexpr float kScale = (ENC == kEncE4M3 && !FULL) ? 0.00390625f : 1.0f;  // 2^-8, exact
@@ -207,7 +209,20 @@ cudaError_t launch_enc(const __half* x, const uint8_t* p, const uint8_t* r, __ha
     // Half-height blocks were measured slower for every Llama-7B shape (the kernel is bound by
     // instruction issue, and they double the MMA and activation-load instructions per weight), so
     // they stay off.
+    // Matrices with few rows (at most one wave of CTAs at three per SM) run with twice the rounds
+    // in flight per lane and two CTAs per SM: measured 10-15 % faster for N = 4096, slower for
+    // the wide layers in full mode.  DPS_STREAM_U2=0|1 overrides (tuning knob).
+    static const int u_forced = [] {
+        const char* e = getenv("DPS_STREAM_U2");
+        return e ? atoi(e) : -1;
+    }();
     constexpr int U = FULL ? 2 : 4;
+    const bool wide_batches = u_forced >= 0 ? u_forced != 0
+                                            : (N + kRowsPerBlock - 1) / kRowsPerBlock <= (int64_t)sm_count() * 3;
+    if (wide_batches) {
+        if (M <= 8) return launch_one<ENC, FULL, 1, 2 * U, false>(x, p, r, y, M, N, K, stream);
+        if (M <= 16) return launch_one<ENC, FULL, 2, 2 * U, false>(x, p, r, y, M, N, K, stream);
+    }
     if (M <= 8) return launch_one<ENC, FULL, 1, U, false>(x, p, r, y, M, N, K, stream);
     if (M <= 16) return launch_one<ENC, FULL, 2, U, false>(x, p, r, y, M, N, K, stream);
     return launch_one<ENC, FULL, 4, U, false>(x, p, r, y, M, N, K, stream);
