@@ -37,26 +37,28 @@ namespace {
 using namespace sm100;
 
 constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
-constexpr int kBlockK = 128;     // K elements per pipeline stage: 128-byte plane rows, the widest swizzled TMA box
-constexpr int kXAtoms = kBlockK / 64;  // the x tile is stored as 64-element (128-byte) swizzle atoms
-constexpr int kACols = kBlockK / 2;    // TMEM columns of one A stage (two FP16 per column)
-constexpr int kAStages = 2;      // A ring in tensor memory when the stage ring has an even depth
-constexpr int kMaxAStages = 3;   // with a 3-deep stage ring every stage has its own A slot
+// K elements per pipeline stage.  128 (128-byte plane rows, the widest swizzled TMA box) for tiles
+// of up to 128 tokens, where the weight stream matters.  64 for 256-token tiles: there the
+// activation tile dominates shared memory (64 KB per 128 K elements) and a ring of two stages
+// cannot cover the load latency; halving the stage doubles the ring depth.
+__host__ __device__ constexpr int block_k(int tn) { return tn >= 256 ? 64 : 128; }
+constexpr int kMaxAStages = 4;   // barrier array size for the A ring in tensor memory
 constexpr int kZipGroups = 2;    // groups of 4 zip warps; group g takes K blocks g, g + G, ...
 constexpr int kThreads = 64 + kZipGroups * 128;
-constexpr int kPlaneStageBytes = kTileRows * kBlockK;  // 16 KB per plane per stage
 constexpr int kMaxStages = 12;
 constexpr int kMaxSplit = 8;     // portable cluster size
-static_assert(kAStages % kZipGroups == 0, "each A stage must belong to one zip group");
 
+__host__ __device__ constexpr int plane_stage_bytes(int tn) { return kTileRows * block_k(tn); }
 __host__ __device__ constexpr int stage_bytes(bool full, int tn) {
-    return kPlaneStageBytes * (full ? 2 : 1) + tn * kBlockK * 2;
+    return plane_stage_bytes(tn) * (full ? 2 : 1) + tn * block_k(tn) * 2;
 }
 // Columns to allocate: accumulator + A ring.  Tiles of up to 64 tokens leave room for three A
 // slots inside 256 columns (two CTAs per SM); wider tiles keep two.
-__host__ __device__ constexpr int a_slots_max(int tn) { return tn <= 64 ? kMaxAStages : kAStages; }
+// A ring with an even stage ring: slots alternate between the zip groups (slot = block % slots).
+__host__ __device__ constexpr int a_slots(int tn) { return tn >= 256 ? 4 : 2; }
+__host__ __device__ constexpr int a_slots_max(int tn) { return tn <= 64 ? 3 : a_slots(tn); }
 __host__ __device__ constexpr int tmem_cols(int tn) {
-    int need = tn + a_slots_max(tn) * kACols;
+    int need = tn + a_slots_max(tn) * (block_k(tn) / 2);
     int c = 32;
     while (c < need) c <<= 1;
     return c;
@@ -118,21 +120,24 @@ struct ZipCtx {
 // Zip loop of one warp: for each of its K blocks, wait for the planes to land and for the A slot
 // to be free, rebuild 128 FP16 weights of this thread's row from the plane bytes and store them
 // into tensor memory.  Returns false if a wait timed out.
-template <int ENC, bool FULL>
+template <int ENC, bool FULL, int TN>
 __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
+    constexpr int kBlockK = block_k(TN);
+    constexpr int kACols = kBlockK / 2;
+    constexpr int kPlaneStageBytes = plane_stage_bytes(TN);
+    constexpr int kSlots = a_slots(TN);
     bool ok = true;
     // Ring positions are advanced incrementally (no division in the loop).  Every stage and every A
     // slot always belongs to the same zip group, so that each waiter sees every phase of the barriers
     // it waits on.  Even ring: blocks alternate between the groups and between two A slots.
     // 3-deep ring: slot = stage, group = stage % groups.
     int s = 0;
-    uint32_t s_parity = 0, pair_parity = 0;   // phase parity of stage s; parity of (i / 2)
-    for (int i = 0; i < z.num_kb && ok;
-         ++i, pair_parity ^= (uint32_t)(i & 1) ^ 1u, s = (s + 1 == z.num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
-        const int a = z.slot_per_stage ? s : (i & 1);
+    uint32_t s_parity = 0;   // phase parity of stage s
+    for (int i = 0; i < z.num_kb && ok; ++i, s = (s + 1 == z.num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
+        const int a = z.slot_per_stage ? s : (i & (kSlots - 1));
         const int owner = z.slot_per_stage ? (s & 1) : (i & 1);
         if (owner != z.group) continue;
-        const uint32_t a_parity = z.slot_per_stage ? s_parity : pair_parity;
+        const uint32_t a_parity = z.slot_per_stage ? s_parity : (uint32_t)(i / kSlots) & 1u;
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(4, i);
         ok = mbar_wait(smem_u32(&z.bar_full[s]), s_parity);
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(5, i);
@@ -145,7 +150,7 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
         uint32_t h[kACols];
 #pragma unroll
         for (int c = 0; c < kBlockK / 16; ++c) {
-            const uint32_t off = ((uint32_t)c ^ z.sw) * 16u;
+            const uint32_t off = ((uint32_t)c ^ z.sw) * 16u;   // sw already reduced for the swizzle width
             uint4 pv, rv = make_uint4(0, 0, 0, 0);
             asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                          : "=r"(pv.x), "=r"(pv.y), "=r"(pv.z), "=r"(pv.w)
@@ -185,6 +190,11 @@ template <int ENC, bool FULL, int TN, bool GROUPED>
 __global__ void __launch_bounds__(kThreads, (tmem_cols(TN) <= 256 ? 2 : 1))
 umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
                    const __grid_constant__ CUtensorMap map_x, const UmmaParams prm, const GroupedParams gp) {
+    constexpr int kBlockK = block_k(TN);
+    constexpr int kXAtoms = kBlockK / 64;    // the x tile is stored as 64-element (128-byte) swizzle atoms
+    constexpr int kACols = kBlockK / 2;      // TMEM columns of one A slot (two FP16 per column)
+    constexpr int kPlaneStageBytes = plane_stage_bytes(TN);
+    constexpr int kSlots = a_slots(TN);
     constexpr int kStage = stage_bytes(FULL, TN);
     constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
     constexpr uint32_t kCols = tmem_cols(TN);
@@ -270,7 +280,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     DPS_CTA_STAMP(1);
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_d = tmem_base;           // TN accumulator columns
-    const uint32_t tmem_a = tmem_base + TN;      // kAStages x kACols columns of packed FP16 pairs
+    const uint32_t tmem_a = tmem_base + TN;      // A ring: slots of kACols columns of packed FP16 pairs
 
     // Split-K sums.  TN <= 64 ("push"): every CTA owns the tokens c with c % split == rank and has a
     // mailbox mail[source rank][slot = c / split][row] in its own shared memory, outside the stage
@@ -331,10 +341,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     } else if (warp == 1) {
         // ---------------- MMA issuer (whole warp converged, one elected lane issues) ----------------
         int s = 0;
-        uint32_t s_parity = 0, pair_parity = 0;
-        for (int i = 0; i < num_kb && ok;
-             ++i, pair_parity ^= (uint32_t)(i & 1) ^ 1u, s = (s + 1 == num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
-            const int a = slot_per_stage ? s : (i & 1);
+        uint32_t s_parity = 0;
+        for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
+            const int a = slot_per_stage ? s : (i & (kSlots - 1));
+            const uint32_t pair_parity = (uint32_t)(i / kSlots) & 1u;
             // The zip warps waited for this stage's TMA loads before they arrived on a_full, so the
             // activation tile of the stage is complete and visible once a_full is: one wait, not two.
             DPS_STAMP(1, i);
@@ -371,13 +381,15 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         zc.num_kb = num_kb; zc.num_stages = num_stages; zc.stage_bytes = kStage;
         zc.slot_per_stage = slot_per_stage;
         zc.smem_base = smem_base; zc.tmem_a = tmem_a; zc.lane_base = lane_base;
-        zc.sw = (uint32_t)(row & 7);  // 128-byte swizzle: 16-byte chunk index ^= row % 8
+        // TMA swizzle of the plane tiles: 128-byte rows: 16-byte chunk index ^= row % 8;
+        // 64-byte rows: chunk index ^= (row / 2) % 4
+        zc.sw = kBlockK == 128 ? (uint32_t)(row & 7) : (uint32_t)((row >> 1) & 3);
         zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
         if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2)) {
             // encoding known only at run time (one per expert): uniform branch per CTA
-            ok = e5m2 ? zip_blocks<kEncE5M2, FULL>(zc) : zip_blocks<kEncE4M3, FULL>(zc);
+            ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN>(zc) : zip_blocks<kEncE4M3, FULL, TN>(zc);
         } else {
-            ok = zip_blocks<ENC, FULL>(zc);
+            ok = zip_blocks<ENC, FULL, TN>(zc);
         }
         // epilogue (first zip group): D[row][token] -> y[token][n0 + row], or -> red for split K
         if (group == 0) {
@@ -583,12 +595,14 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         configured = true;
     }
     CUtensorMap mp, mr, mx;
+    constexpr int kBlockK = block_k(TN);
+    constexpr CUtensorMapSwizzle kPlaneSwizzle = kBlockK == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
     if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, (uint64_t)K, kTileRows, kBlockK,
-                     CU_TENSOR_MAP_SWIZZLE_128B))
+                     kPlaneSwizzle))
         return cudaErrorInvalidValue;
     if (FULL) {
         if (!make_map_2d(&mr, r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, (uint64_t)K, kTileRows, kBlockK,
-                         CU_TENSOR_MAP_SWIZZLE_128B))
+                         kPlaneSwizzle))
             return cudaErrorInvalidValue;
     } else {
         mr = mp;
@@ -703,6 +717,8 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
         configured = true;
     }
     CUtensorMap mp, mr, mx;
+    constexpr int kBlockK = block_k(TN);
+    static_assert(kBlockK == 128, "grouped launches use tiles of at most 128 tokens");
     if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows,
                      kBlockK, CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
