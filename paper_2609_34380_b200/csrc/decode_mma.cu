@@ -64,7 +64,7 @@ __device__ __forceinline__ void to_half_pairs(const uint4& p, const uint4& r, ui
 // HALF: the CTA owns 8 weight rows instead of 16 (the upper half of every MMA tile is zero).  It
 // doubles the number of CTAs for matrices with few rows; the MMA work wasted is irrelevant here.
 template <int ENC, bool FULL, int NT, int U, bool HALF>
-__global__ void __launch_bounds__(kThreads, (U * (FULL ? 2 : 1) >= 8 ? 2 : 3))
+__global__ void __launch_bounds__(kThreads, 2)
 decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, const uint8_t* __restrict__ Rp,
                   __half* __restrict__ y, int M, int64_t N, int64_t K) {
     constexpr float kScale = (ENC == kEncE4M3 && !FULL) ? 0.00390625f : 1.0f;  // 2^-8, exact
@@ -98,8 +98,18 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[n][c] = 0.f;
 
+        auto load_x = [&](uint4 (&xb)[NT][2], int koff, bool in) {
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                xb[n][0] = xb[n][1] = make_uint4(0, 0, 0, 0);
+                if (in) {
+                    xb[n][0] = *reinterpret_cast<const uint4*>(xrow[n] + koff);
+                    xb[n][1] = *reinterpret_cast<const uint4*>(xrow[n] + koff + 8);
+                }
+            }
+        };
         auto multiply = [&](const uint4& wp_lo, const uint4& wp_hi, const uint4& wr_lo, const uint4& wr_hi,
-                            int koff, bool in) {
+                            const uint4 (&xb)[NT][2]) {
             uint32_t a_lo[8], a_hi[8];
             to_half_pairs<ENC, FULL>(wp_lo, wr_lo, a_lo);
             if (HALF) {
@@ -110,11 +120,7 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
             }
 #pragma unroll
             for (int n = 0; n < NT; ++n) {
-                uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;
-                if (in) {
-                    b0 = *reinterpret_cast<const uint4*>(xrow[n] + koff);
-                    b1 = *reinterpret_cast<const uint4*>(xrow[n] + koff + 8);
-                }
+                const uint4 b0 = xb[n][0], b1 = xb[n][1];
                 const uint32_t bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
                 // MMA j takes bytes 4j..4j+3 of the lane's 16: K slots (2t, 2t+1) <- pair 2j and
                 // K slots (2t+8, 2t+9) <- pair 2j+1, for the weights and the activations alike.
@@ -139,8 +145,13 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
                     if (!HALF) wr_hi[u] = ldg_stream(r_hi + base + u * kRoundK);
                 }
             }
+            // the activation fragments of the batch are fetched together with the weights, so that
+            // their (L1 / L2) latency hides behind the DRAM latency of the weight loads
+            uint4 xb[U][NT][2];
 #pragma unroll
-            for (int u = 0; u < U; ++u) multiply(wp_lo[u], wp_hi[u], wr_lo[u], wr_hi[u], base + u * kRoundK, true);
+            for (int u = 0; u < U; ++u) load_x(xb[u], base + u * kRoundK, true);
+#pragma unroll
+            for (int u = 0; u < U; ++u) multiply(wp_lo[u], wp_hi[u], wr_lo[u], wr_hi[u], xb[u]);
         }
         for (; r0 < full_rounds + (has_tail ? 1 : 0); ++r0) {   // leftover rounds and the ragged end of K
             const int base = r0 * kRoundK;
@@ -155,7 +166,9 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
                     if (!HALF) wr_hi = ldg_stream(r_hi + base);
                 }
             }
-            multiply(wp_lo, wp_hi, wr_lo, wr_hi, base, in);
+            uint4 xb[NT][2];
+            load_x(xb, base, in);
+            multiply(wp_lo, wp_hi, wr_lo, wr_hi, xb);
         }
         // accumulator fragment: c0,c1 = (row g, tokens 2t, 2t+1), c2,c3 = (row g+8, same tokens)
 #pragma unroll

@@ -37,28 +37,31 @@ namespace {
 using namespace sm100;
 
 constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
-// K elements per pipeline stage.  128 (128-byte plane rows, the widest swizzled TMA box) for tiles
-// of up to 128 tokens, where the weight stream matters.  64 for 256-token tiles: there the
-// activation tile dominates shared memory (64 KB per 128 K elements) and a ring of two stages
-// cannot cover the load latency; halving the stage doubles the ring depth.
-__host__ __device__ constexpr int block_k(int tn) { return tn >= 256 ? 64 : 128; }
+// K elements per pipeline stage.  128 (128-byte plane rows, the widest swizzled TMA box) where it
+// still leaves a ring of at least three or four stages.  64 where it does not: 256-token tiles (the
+// activation tile alone is 64 KB per 128 K elements) and full mode with small tiles (two planes
+// per stage).  A ring of two stages cannot cover the 1600-2150 cycles a stage load takes;
+// halving the stage doubles the ring depth.
+__host__ __device__ constexpr int block_k(bool full, int tn) { return (tn >= 256 || (full && tn <= 64)) ? 64 : 128; }
 constexpr int kMaxAStages = 4;   // barrier array size for the A ring in tensor memory
 constexpr int kZipGroups = 2;    // groups of 4 zip warps; group g takes K blocks g, g + G, ...
 constexpr int kThreads = 64 + kZipGroups * 128;
 constexpr int kMaxStages = 12;
 constexpr int kMaxSplit = 8;     // portable cluster size
 
-__host__ __device__ constexpr int plane_stage_bytes(int tn) { return kTileRows * block_k(tn); }
+__host__ __device__ constexpr int plane_stage_bytes(bool full, int tn) { return kTileRows * block_k(full, tn); }
 __host__ __device__ constexpr int stage_bytes(bool full, int tn) {
-    return plane_stage_bytes(tn) * (full ? 2 : 1) + tn * block_k(tn) * 2;
+    return plane_stage_bytes(full, tn) * (full ? 2 : 1) + tn * block_k(full, tn) * 2;
 }
 // Columns to allocate: accumulator + A ring.  Tiles of up to 64 tokens leave room for three A
 // slots inside 256 columns (two CTAs per SM); wider tiles keep two.
 // A ring with an even stage ring: slots alternate between the zip groups (slot = block % slots).
-__host__ __device__ constexpr int a_slots(int tn) { return tn >= 256 ? 4 : 2; }
-__host__ __device__ constexpr int a_slots_max(int tn) { return tn <= 64 ? 3 : a_slots(tn); }
-__host__ __device__ constexpr int tmem_cols(int tn) {
-    int need = tn + a_slots_max(tn) * (block_k(tn) / 2);
+__host__ __device__ constexpr int a_slots(bool full, int tn) { return block_k(full, tn) == 64 ? 4 : 2; }
+__host__ __device__ constexpr int a_slots_max(bool full, int tn) {
+    return (tn <= 64 && a_slots(full, tn) < 3) ? 3 : a_slots(full, tn);
+}
+__host__ __device__ constexpr int tmem_cols(bool full, int tn) {
+    int need = tn + a_slots_max(full, tn) * (block_k(full, tn) / 2);
     int c = 32;
     while (c < need) c <<= 1;
     return c;
@@ -122,10 +125,10 @@ struct ZipCtx {
 // into tensor memory.  Returns false if a wait timed out.
 template <int ENC, bool FULL, int TN>
 __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
-    constexpr int kBlockK = block_k(TN);
+    constexpr int kBlockK = block_k(FULL, TN);
     constexpr int kACols = kBlockK / 2;
-    constexpr int kPlaneStageBytes = plane_stage_bytes(TN);
-    constexpr int kSlots = a_slots(TN);
+    constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN);
+    constexpr int kSlots = a_slots(FULL, TN);
     bool ok = true;
     // Ring positions are advanced incrementally (no division in the loop).  Every stage and every A
     // slot always belongs to the same zip group, so that each waiter sees every phase of the barriers
@@ -187,17 +190,17 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
 
 // ENC == 0 (grouped launches only): the encoding is a per-expert run-time value.
 template <int ENC, bool FULL, int TN, bool GROUPED>
-__global__ void __launch_bounds__(kThreads, (tmem_cols(TN) <= 256 ? 2 : 1))
+__global__ void __launch_bounds__(kThreads, (tmem_cols(FULL, TN) <= 256 ? 2 : 1))
 umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
                    const __grid_constant__ CUtensorMap map_x, const UmmaParams prm, const GroupedParams gp) {
-    constexpr int kBlockK = block_k(TN);
+    constexpr int kBlockK = block_k(FULL, TN);
     constexpr int kXAtoms = kBlockK / 64;    // the x tile is stored as 64-element (128-byte) swizzle atoms
     constexpr int kACols = kBlockK / 2;      // TMEM columns of one A slot (two FP16 per column)
-    constexpr int kPlaneStageBytes = plane_stage_bytes(TN);
-    constexpr int kSlots = a_slots(TN);
+    constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN);
+    constexpr int kSlots = a_slots(FULL, TN);
     constexpr int kStage = stage_bytes(FULL, TN);
     constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
-    constexpr uint32_t kCols = tmem_cols(TN);
+    constexpr uint32_t kCols = tmem_cols(FULL, TN);
     constexpr uint32_t kIdesc = umma_idesc_f16(kTileRows, TN);
 
     extern __shared__ uint8_t smem_raw[];
@@ -536,7 +539,7 @@ template <int ENC, bool FULL, int TN>
 cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y, int64_t M, int64_t N, int64_t K,
                       int* status, cudaStream_t stream) {
     constexpr int kStage = stage_bytes(FULL, TN);
-    constexpr int kCtasPerSm = tmem_cols(TN) <= 256 ? 2 : 1;
+    constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
     constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
     constexpr int kMailMax = TN <= 64 ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox, worst case
     // Ring depth for a given mailbox size: even, or exactly 3 (every stage then owns an A slot,
@@ -553,7 +556,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         int d = (smem_total - mail_bytes) / kStage;
         if (d > 8) d = 8;
         if (d < 2) d = 2;
-        if (d % kZipGroups != 0 && !(d == 3 && a_slots_max(TN) >= 3)) d -= d % kZipGroups;
+        if (d % kZipGroups != 0 && !(d == 3 && a_slots_max(FULL, TN) >= 3)) d -= d % kZipGroups;
         return d;
     };
     const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kMailMax + 1024;
@@ -595,7 +598,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         configured = true;
     }
     CUtensorMap mp, mr, mx;
-    constexpr int kBlockK = block_k(TN);
+    constexpr int kBlockK = block_k(FULL, TN);
     constexpr CUtensorMapSwizzle kPlaneSwizzle = kBlockK == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
     if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, (uint64_t)K, kTileRows, kBlockK,
                      kPlaneSwizzle))
@@ -699,7 +702,7 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
                               const int32_t* num_tiles, const int32_t* sorted_rows, int max_tiles, int* status,
                               cudaStream_t stream) {
     constexpr int kStage = stage_bytes(FULL, TN);
-    constexpr int kCtasPerSm = tmem_cols(TN) <= 256 ? 2 : 1;
+    constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
     constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
     int stages = kSmemTotal / kStage;
     if (stages > 8) stages = 8;
@@ -717,14 +720,14 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
         configured = true;
     }
     CUtensorMap mp, mr, mx;
-    constexpr int kBlockK = block_k(TN);
-    static_assert(kBlockK == 128, "grouped launches use tiles of at most 128 tokens");
+    constexpr int kBlockK = block_k(FULL, TN);
+    constexpr CUtensorMapSwizzle kPlaneSwizzle = kBlockK == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
     if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows,
-                     kBlockK, CU_TENSOR_MAP_SWIZZLE_128B))
+                     kBlockK, kPlaneSwizzle))
         return cudaErrorInvalidValue;
     if (FULL) {
         if (!make_map_2d(&mr, r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows,
-                         kBlockK, CU_TENSOR_MAP_SWIZZLE_128B))
+                         kBlockK, kPlaneSwizzle))
             return cudaErrorInvalidValue;
     } else {
         mr = mp;
