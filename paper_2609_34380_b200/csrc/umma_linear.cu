@@ -38,11 +38,18 @@ using namespace sm100;
 
 constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
 // K elements per pipeline stage.  128 (128-byte plane rows, the widest swizzled TMA box) where it
-// still leaves a ring of at least three or four stages.  64 where it does not: 256-token tiles (the
-// activation tile alone is 64 KB per 128 K elements) and full mode with small tiles (two planes
-// per stage).  A ring of two stages cannot cover the 1600-2150 cycles a stage load takes;
-// halving the stage doubles the ring depth.
-__host__ __device__ constexpr int block_k(bool full, int tn) { return (tn >= 256 || (full && tn <= 64)) ? 64 : 128; }
+// still leaves a ring of at least three or four stages: fast mode with tiles of up to 64 tokens.
+// 64 where it does not: tiles of 128 tokens and more (the activation tile alone is 32-64 KB per
+// 128 K elements) and full mode with small tiles (two planes per stage).  A ring of two stages
+// cannot cover the 1600-2150 cycles a stage load takes; halving the stage doubles the ring depth.
+// Measured: 64 everywhere costs fast-mode decode 10-20 % (64-byte plane rows stream worse), 128
+// everywhere costs full mode and the grouped kernel about as much.
+#ifndef DPS_BK64_FROM
+#define DPS_BK64_FROM 128
+#endif
+__host__ __device__ constexpr int block_k(bool full, int tn) {
+    return (tn >= DPS_BK64_FROM || (full && tn <= 64)) ? 64 : 128;
+}
 constexpr int kMaxAStages = 4;   // barrier array size for the A ring in tensor memory
 constexpr int kZipGroups = 2;    // groups of 4 zip warps; group g takes K blocks g, g + G, ...
 constexpr int kThreads = 64 + kZipGroups * 128;
