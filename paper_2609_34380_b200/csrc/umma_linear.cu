@@ -150,12 +150,11 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
         const uint32_t a_parity = z.slot_per_stage ? s_parity : (uint32_t)(i / kSlots) & 1u;
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(4, i);
         ok = mbar_wait(smem_u32(&z.bar_full[s]), s_parity);
-        if (z.warp == 2 + 4 * z.group) DPS_STAMP(5, i);
-        if (ok) ok = mbar_wait(smem_u32(&z.bar_a_empty[a]), a_parity ^ 1u);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
-        if (z.warp == 2 + 4 * z.group) DPS_STAMP(6, i);
-        tc_fence_after_sync();
+        if (z.warp == 2 + 4 * z.group) DPS_STAMP(5, i);
+        // Read and rebuild the weights FIRST, into registers: that needs the stage, not the A slot,
+        // so it overlaps the MMAs that are still reading the slot's previous contents.
         const uint32_t prow = z.smem_base + (uint32_t)s * z.stage_bytes + (uint32_t)z.row * kBlockK;
         uint32_t h[kACols];
 #pragma unroll
@@ -175,6 +174,11 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) h[c * 8 + j] = h8[j];
         }
+        ok = mbar_wait(smem_u32(&z.bar_a_empty[a]), a_parity ^ 1u);   // now the slot must be free
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+        if (z.warp == 2 + 4 * z.group) DPS_STAMP(6, i);
+        tc_fence_after_sync();
 #pragma unroll
         for (int t = 0; t < kACols / 32; ++t) {
             uint32_t part[32];

@@ -175,3 +175,51 @@ def test_launch_counter_moves():
     x = workloads.activations(1, 64, 52, device=DEV)
     dps.dps_linear(dps.DPS_MODE_FULL, enc, x, p, r)
     assert dps.dps_launch_count() > before
+
+
+def test_inf_and_nan_weights_follow_the_bit_rule():
+    """Inf / NaN weights force E5M2; split and reconstruction stay bit-exact, and the products carry
+    the same non-finite pattern as the oracle's (a NaN whose payload sits only in the low mantissa
+    byte turns into Inf in fast mode: that is what dropping the residual means)."""
+    N, K = 64, 256
+    w = workloads.weights(N, K, 61).clone()
+    words = to_np_words(w).copy()
+    words[3, 7] = 0x7C00      # +inf
+    words[5, 9] = 0xFC00      # -inf
+    words[8, 1] = 0x7E01      # NaN, payload in both bytes
+    words[9, 2] = 0x7C01      # NaN whose payload is in the residual byte only
+    w = torch.from_numpy(words.view(np.int16)).view(torch.float16).to(DEV)
+    p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+    assert enc == dps.DPS_ENC_E5M2
+    p_ref, r_ref, _ = oracle.split(words, oracle.ENC_E5M2)
+    assert np.array_equal(to_np_bytes(p), p_ref) and np.array_equal(to_np_bytes(r), r_ref)
+    assert np.array_equal(to_np_words(dps.dps_reconstruct(p, r, enc)), words)
+    for M in (1, 8, 40):
+        x = workloads.activations(M, K, 62, device=DEV).abs() + 0.5      # no zeros: inf * x stays inf
+        for mode in MODES:
+            y = y_as_f64(dps.dps_linear(mode, enc, x, p, r if mode else None))
+            with np.errstate(invalid="ignore", over="ignore"):
+                ref = oracle.linear(mode, enc, to_np_words(x), p_ref, r_ref)
+            assert np.array_equal(np.isnan(y), np.isnan(ref)), (M, mode)
+            assert np.array_equal(np.isinf(y), np.isinf(ref)), (M, mode)
+            assert np.array_equal(np.sign(y[np.isinf(y)]), np.sign(ref[np.isinf(ref)]))
+            fin = np.isfinite(ref)
+            assert np.max(np.abs(y[fin] - ref[fin])) <= 2e-3 * np.max(np.abs(ref[fin]))
+            assert np.isinf(ref[:, 9]).all() if mode == dps.DPS_MODE_FAST else np.isnan(ref[:, 9]).all()
+
+
+def test_randomised_shapes_modes_and_encodings():
+    """Seeded sweep over awkward shapes: every kernel family and dispatch boundary sees ragged
+    N (multiples of 8), ragged K (multiples of 16) and token counts on both sides of each threshold."""
+    rng = np.random.default_rng(20261125)
+    token_pool = [1, 2, 5, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 200, 256, 257, 300, 513]
+    for case in range(36):
+        N = int(rng.integers(1, 400)) * 8
+        K = int(rng.integers(1, 380)) * 16
+        M = int(token_pool[int(rng.integers(0, len(token_pool)))])
+        enc_req = ENCS[int(rng.integers(0, 2))]
+        mode = MODES[int(rng.integers(0, 2))]
+        _, p, r, enc = planes(N, K, 7000 + case, enc_req)
+        x = workloads.activations(M, K, 8000 + case, device=DEV)
+        run_and_check(mode, enc, x, p, r, f"random case {case}: M={M} N={N} K={K} mode={mode} enc={enc}")
+    assert dps.dps_stream_status() == dps.DPS_OK
