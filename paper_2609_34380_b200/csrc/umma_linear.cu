@@ -39,13 +39,13 @@ using namespace sm100;
 constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
 // K elements per pipeline stage.  128 (128-byte plane rows, the widest swizzled TMA box) where it
 // still leaves a ring of at least three or four stages: fast mode with tiles of up to 64 tokens.
-// 64 where it does not: tiles of 128 tokens and more (the activation tile alone is 32-64 KB per
+// 64 where it does not: tiles of 96 tokens and more (the activation tile alone is 32-64 KB per
 // 128 K elements) and full mode with small tiles (two planes per stage).  A ring of two stages
 // cannot cover the 1600-2150 cycles a stage load takes; halving the stage doubles the ring depth.
 // Measured: 64 everywhere costs fast-mode decode 10-20 % (64-byte plane rows stream worse), 128
 // everywhere costs full mode and the grouped kernel about as much.
 #ifndef DPS_BK64_FROM
-#define DPS_BK64_FROM 128
+#define DPS_BK64_FROM 96
 #endif
 __host__ __device__ constexpr int block_k(bool full, int tn) {
     return (tn >= DPS_BK64_FROM || (full && tn <= 64)) ? 64 : 128;
@@ -778,9 +778,14 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
 
 }  // namespace
 
+// Token-tile width of grouped launches: wide enough that an expert with 1.5 times the average
+// number of rows still fits one tile (its planes are then streamed once), no wider than needed
+// (every tile drags TN activation rows through L2 per weight block: at 128 tokens that is twice
+// the plane bytes, and L2-to-SM bandwidth, not HBM, becomes the limit).
 int grouped_tile_tokens(int64_t A, int32_t E) {
-    const int64_t target = 2 * ((A + E - 1) / E);
-    return target <= 16 ? 16 : target <= 32 ? 32 : target <= 64 ? 64 : 128;
+    const int64_t avg = (A + E - 1) / E;
+    const int64_t target = avg + (avg + 1) / 2;
+    return target <= 16 ? 16 : target <= 32 ? 32 : target <= 64 ? 64 : target <= 96 ? 96 : 128;
 }
 
 cudaError_t launch_umma_grouped(int mode, const uint32_t* e5m2_mask, const void* x_sorted, const uint8_t* p,
@@ -797,6 +802,7 @@ cudaError_t launch_umma_grouped(int mode, const uint32_t* e5m2_mask, const void*
     DPS_GROUPED_CASE(16)
     DPS_GROUPED_CASE(32)
     DPS_GROUPED_CASE(64)
+    DPS_GROUPED_CASE(96)
     DPS_GROUPED_CASE(128)
 #undef DPS_GROUPED_CASE
     return cudaErrorInvalidValue;
