@@ -51,8 +51,11 @@ __host__ __device__ constexpr int block_k(bool full, int tn) {
     return (tn >= DPS_BK64_FROM || (full && tn <= 64)) ? 64 : 128;
 }
 constexpr int kMaxAStages = 4;   // barrier array size for the A ring in tensor memory
-constexpr int kZipGroups = 2;    // groups of 4 zip warps; group g takes K blocks g, g + G, ...
-constexpr int kThreads = 64 + kZipGroups * 128;
+// Groups of 4 zip warps; group g takes K blocks g, g + G, ...  Two groups everywhere: four were
+// measured for 256-token full-mode tiles (one CTA per SM) and changed nothing -- once the stage
+// ring is four deep the zip warps no longer hold the tensor pipe back there.
+__host__ __device__ constexpr int zip_groups(bool full, int tn) { return (full && tn >= 100000) ? 4 : 2; }
+__host__ __device__ constexpr int cta_threads(bool full, int tn) { return 64 + zip_groups(full, tn) * 128; }
 constexpr int kMaxStages = 12;
 constexpr int kMaxSplit = 8;     // portable cluster size
 
@@ -145,7 +148,7 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
     uint32_t s_parity = 0;   // phase parity of stage s
     for (int i = 0; i < z.num_kb && ok; ++i, s = (s + 1 == z.num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
         const int a = z.slot_per_stage ? s : (i & (kSlots - 1));
-        const int owner = z.slot_per_stage ? (s & 1) : (i & 1);
+        const int owner = z.slot_per_stage ? (s & 1) : (i & (zip_groups(FULL, TN) - 1));
         if (owner != z.group) continue;
         const uint32_t a_parity = z.slot_per_stage ? s_parity : (uint32_t)(i / kSlots) & 1u;
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(4, i);
@@ -201,7 +204,7 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
 
 // ENC == 0 (grouped launches only): the encoding is a per-expert run-time value.
 template <int ENC, bool FULL, int TN, bool GROUPED>
-__global__ void __launch_bounds__(kThreads, (tmem_cols(FULL, TN) <= 256 ? 2 : 1))
+__global__ void __launch_bounds__(cta_threads(FULL, TN), (tmem_cols(FULL, TN) <= 256 ? 2 : 1))
 umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
                    const __grid_constant__ CUtensorMap map_x, const UmmaParams prm, const GroupedParams gp) {
     constexpr int kBlockK = block_k(FULL, TN);
@@ -235,6 +238,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_stages = prm.num_stages;
+    constexpr int kZipGroups = zip_groups(FULL, TN);
+    constexpr int kThreads = cta_threads(FULL, TN);
     const bool slot_per_stage = (num_stages % kZipGroups) != 0;   // only the 3-deep ring
     // Tile order (dense launches with several token tiles): CTAs are handed out x-fastest, so walk
     // groups of 8 row tiles x all token tiles.  The CTAs running at any moment then share 8 row
@@ -550,6 +555,8 @@ template <int ENC, bool FULL, int TN>
 cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y, int64_t M, int64_t N, int64_t K,
                       int* status, cudaStream_t stream) {
     constexpr int kStage = stage_bytes(FULL, TN);
+    constexpr int kZipGroups = zip_groups(FULL, TN);
+    constexpr int kThreads = cta_threads(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
     constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
     constexpr int kMailMax = TN <= 64 ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox, worst case
@@ -567,7 +574,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         int d = (smem_total - mail_bytes) / kStage;
         if (d > 8) d = 8;
         if (d < 2) d = 2;
-        if (d % kZipGroups != 0 && !(d == 3 && a_slots_max(FULL, TN) >= 3)) d -= d % kZipGroups;
+        if (d % kZipGroups != 0 && !(d == 3 && kZipGroups == 2 && a_slots_max(FULL, TN) >= 3)) d -= d % kZipGroups;
         return d;
     };
     const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kMailMax + 1024;
@@ -713,6 +720,8 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
                               const int32_t* num_tiles, const int32_t* sorted_rows, int max_tiles, int* status,
                               cudaStream_t stream) {
     constexpr int kStage = stage_bytes(FULL, TN);
+    constexpr int kZipGroups = zip_groups(FULL, TN);
+    constexpr int kThreads = cta_threads(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
     constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
     int stages = kSmemTotal / kStage;
