@@ -54,7 +54,7 @@ constexpr int kMaxAStages = 4;   // barrier array size for the A ring in tensor 
 // Groups of 4 zip warps; group g takes K blocks g, g + G, ...  Two groups everywhere: four were
 // measured for 256-token full-mode tiles (one CTA per SM) and changed nothing -- once the stage
 // ring is four deep the zip warps no longer hold the tensor pipe back there.
-__host__ __device__ constexpr int zip_groups(bool full, int tn) { return (full && tn >= 100000) ? 4 : 2; }
+__host__ __device__ constexpr int zip_groups(bool /*full*/, int /*tn*/) { return 2; }
 __host__ __device__ constexpr int cta_threads(bool full, int tn) { return 64 + zip_groups(full, tn) * 128; }
 constexpr int kMaxStages = 12;
 constexpr int kMaxSplit = 8;     // portable cluster size
