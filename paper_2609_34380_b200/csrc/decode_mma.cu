@@ -63,13 +63,34 @@ __device__ __forceinline__ void to_half_pairs(const uint4& p, const uint4& r, ui
 
 // HALF: the CTA owns 8 weight rows instead of 16 (the upper half of every MMA tile is zero).  It
 // doubles the number of CTAs for matrices with few rows; the MMA work wasted is irrelevant here.
+// Three CTAs per SM for the variant that fits them (full mode, 8 tokens, two rounds in flight:
+// 80 registers); one register more and the allocation granularity drops it to two CTAs, which
+// was measured 10 % slower on the wide Llama-7B layers.
 template <int ENC, bool FULL, int NT, int U, bool HALF>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, (FULL && NT == 1 && U == 2) ? 3 : 2)
 decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, const uint8_t* __restrict__ Rp,
-                  __half* __restrict__ y, int M, int64_t N, int64_t K) {
+                  __half* __restrict__ y, int M, int64_t N, int64_t K, int prefetch_steps,
+                  int prefetch_ctas) {
     constexpr float kScale = (ENC == kEncE4M3 && !FULL) ? 0.00390625f : 1.0f;  // 2^-8, exact
     __shared__ float red[kWarps][kRowsPerBlock][NT * 8 + 1];
     sm100::grid_launch_dependents();
+    // A CTA that becomes resident while the preceding kernel drains has nothing to compute with yet
+    // (its activations are that kernel's output), but its weights are model state: ask L2 for the
+    // CTA's row block now, so that the DRAM pipe keeps working through the other kernel's tail and
+    // the loads below hit L2.  Thread i takes row i / 16 and every 16th 128-byte line of it.
+    if (prefetch_steps > 0 && (int)blockIdx.x < prefetch_ctas) {
+        const int64_t prow = (int64_t)blockIdx.x * (HALF ? 8 : kRowsPerBlock) + (threadIdx.x >> 4);
+        if (prow < N && (!HALF || (threadIdx.x >> 4) < 8)) {
+            const int64_t pbase = prow * K + (threadIdx.x & 15) * 128;
+            for (int j = 0; j < prefetch_steps; ++j) {
+                const int64_t off = (int64_t)j * 2048 + (threadIdx.x & 15) * 128;
+                if (off < K) {
+                    sm100::prefetch_l2(P + pbase + (int64_t)j * 2048);
+                    if (FULL) sm100::prefetch_l2(Rp + pbase + (int64_t)j * 2048);
+                }
+            }
+        }
+    }
     sm100::grid_dependency_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -153,22 +174,35 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
 #pragma unroll
             for (int u = 0; u < U; ++u) multiply(wp_lo[u], wp_hi[u], wr_lo[u], wr_hi[u], xb[u]);
         }
-        for (; r0 < full_rounds + (has_tail ? 1 : 0); ++r0) {   // leftover rounds and the ragged end of K
-            const int base = r0 * kRoundK;
-            if ((int64_t)base + warp * 64 >= K) continue;       // warp-uniform: the MMA needs the whole warp
-            const bool in = (int64_t)base + kl < K;
-            uint4 wp_lo = make_uint4(0, 0, 0, 0), wp_hi = wp_lo, wr_lo = wp_lo, wr_hi = wp_lo;
-            if (in) {
-                wp_lo = ldg_stream(p_lo + base);
-                if (!HALF) wp_hi = ldg_stream(p_hi + base);
-                if (FULL) {
-                    wr_lo = ldg_stream(r_lo + base);
-                    if (!HALF) wr_hi = ldg_stream(r_hi + base);
+        const int total_rounds = full_rounds + (has_tail ? 1 : 0);
+        // Leftover rounds and the ragged end of K: predicated batches (of at most 128 bytes per lane, which
+        // keeps the predicated copy of the loop body free of register spills), never one round at
+        // a time -- a lone round costs a full DRAM latency.
+        constexpr int UT = FULL ? 2 : (U > 4 ? 4 : U);
+        for (; r0 < total_rounds; r0 += UT) {
+            uint4 wp_lo[UT], wp_hi[UT], wr_lo[UT], wr_hi[UT];
+            uint4 xb[UT][NT][2];
+#pragma unroll
+            for (int u = 0; u < UT; ++u) {
+                const int base = (r0 + u) * kRoundK;
+                const bool in = r0 + u < total_rounds && (int64_t)base + kl < K;
+                wp_lo[u] = wp_hi[u] = wr_lo[u] = wr_hi[u] = make_uint4(0, 0, 0, 0);
+                if (in) {
+                    wp_lo[u] = ldg_stream(p_lo + base);
+                    if (!HALF) wp_hi[u] = ldg_stream(p_hi + base);
+                    if (FULL) {
+                        wr_lo[u] = ldg_stream(r_lo + base);
+                        if (!HALF) wr_hi[u] = ldg_stream(r_hi + base);
+                    }
                 }
+                load_x(xb[u], base, in);
             }
-            uint4 xb[NT][2];
-            load_x(xb, base, in);
-            multiply(wp_lo, wp_hi, wr_lo, wr_hi, xb);
+#pragma unroll
+            for (int u = 0; u < UT; ++u) {
+                // warp-uniform skip (the MMA needs the whole warp); lanes past K multiply zeros
+                const bool warp_in = r0 + u < total_rounds && (int64_t)(r0 + u) * kRoundK + warp * 64 < K;
+                if (warp_in) multiply(wp_lo[u], wp_hi[u], wr_lo[u], wr_hi[u], xb[u]);
+            }
         }
         // accumulator fragment: c0,c1 = (row g, tokens 2t, 2t+1), c2,c3 = (row g+8, same tokens)
 #pragma unroll
@@ -210,7 +244,20 @@ cudaError_t launch_one(const __half* x, const uint8_t* p, const uint8_t* r, __ha
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_mma_kernel<ENC, FULL, NT, U, HALF>, x, p, r, y, M, N, K);
+    // DPS_STREAM_PREFETCH=<steps> overrides how many 2 KB column steps of its row block a CTA asks
+    // L2 for before it waits for the preceding kernel (0 = none), DPS_STREAM_PREFETCH_CTAS how many
+    // CTAs of the grid do so.  Measured on Llama-7B shapes: one step by the first wave of CTAs gains
+    // 1-10 %; whole row blocks, or every CTA of a grid of several waves, lose.
+    static const int prefetch_steps = [] {
+        const char* e = getenv("DPS_STREAM_PREFETCH");
+        return e ? atoi(e) : 1;
+    }();
+    static const int prefetch_ctas = [] {
+        const char* e = getenv("DPS_STREAM_PREFETCH_CTAS");
+        return e ? atoi(e) : 2 * sm_count();
+    }();
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_mma_kernel<ENC, FULL, NT, U, HALF>, x, p, r, y, M, N, K,
+                                       prefetch_steps, prefetch_ctas);
     count_launch();
     return e;
 }

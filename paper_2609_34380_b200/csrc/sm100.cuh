@@ -201,6 +201,11 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
 // launch_dependents: the next kernel in the stream (if launched with programmatic stream
 // serialization) may begin once every CTA of this grid has executed this or exited.
 // wait: blocks until the preceding grid has completed and its memory operations are visible.
+// Ask for one line of global memory to be brought into L2.  L2 is the point of coherence for this
+// GPU's own writes, so a line requested before an earlier kernel has finished writing it is still
+// read correctly afterwards.
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 __device__ __forceinline__ void grid_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
