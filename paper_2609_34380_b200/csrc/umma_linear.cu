@@ -540,14 +540,13 @@ bool make_map_2d(CUtensorMap* map, const void* base, CUtensorMapDataType dt, int
 // K split for a launch of `tiles` output tiles.  capacity[s] = CTAs that can be resident at once
 // when launched as clusters of s (clusters must fit inside one GPC, so this is not a multiple of
 // the SM count).  Measured on B200: a second wave costs more than it buys, so take the largest
-// factor (<= 8, a portable cluster) whose CTAs are (all but a few per cent) resident at once,
-// keeping at least 4 K blocks per CTA.  The 10 % allowance lets 32 row tiles take a split of 8
-// (256 CTAs against a packing estimate of 240), measured 5-11 % faster than 6.
+// factor (<= 8, a portable cluster) whose CTAs are all resident at once, keeping at least 4 K
+// blocks per CTA.
 int choose_split(int64_t tiles, int total_kb, const int* capacity) {
     int best = 1;
     for (int s = 2; s <= kMaxSplit; ++s) {
         if (total_kb / s < 4) break;
-        if (tiles * s * 10 <= (int64_t)capacity[s] * 11) best = s;
+        if (tiles * s <= capacity[s]) best = s;
     }
     return best;
 }
@@ -614,6 +613,12 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         if (capacity[1] <= 0) capacity[1] = slots;
         const int base = capacity[1];
         for (int s = 1; s <= kMaxSplit; ++s) capacity[s] = (int)((int64_t)capacity[s] * slots / base);
+        // With two CTAs per SM a cluster of even size s needs only s / 2 SMs of a GPC, so it packs
+        // like a cluster of s / 2 at one CTA per SM (32 row tiles split 8 ways, 256 CTAs, were
+        // measured 5-11 % faster than split 6 ways, which the plain rescaling would have chosen).
+        if (kCtasPerSm == 2)
+            for (int s = kMaxSplit; s >= 2; s -= 2)
+                if (capacity[s / 2] > capacity[s]) capacity[s] = capacity[s / 2];
         configured = true;
     }
     CUtensorMap mp, mr, mx;
