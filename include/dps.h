@@ -21,6 +21,13 @@
  *     contiguous; y[M][N] = x[M][K] * W^T.  x and y are IEEE binary16, row-major.
  *   - The persistent plane P and the residual plane R are SEPARATE allocations of N*K
  *     bytes each, index-for-index identical to W.
+ *   - The planes are MODEL STATE.  The linear kernels start fetching them while the
+ *     kernel that precedes the call on the stream is still draining (programmatic
+ *     dependent launch); only the activations wait for that kernel.  So a plane must not
+ *     be written by the kernel launched immediately before dps_linear / dps_moe_linear
+ *     on the same stream.  Planes written by dps_split_weights, by a copy
+ *     (cudaMemcpyAsync) or by any kernel further back in the stream are safe:
+ *     dps_split_weights ends with a fence launch for exactly this reason.
  *   - Pointers are DEVICE pointers unless a parameter says "host".  The caller owns
  *     every buffer; the library never allocates or frees device memory.
  *   - cuda_stream is a cudaStream_t passed as void* (NULL = the default stream).  Work

@@ -78,6 +78,12 @@ int stream_grid(int64_t items) {
     return (int)(blocks < cap ? (blocks > 0 ? blocks : 1) : cap);
 }
 
+// Empty kernel launched (as an ordinary, fully ordered launch) after the planes have been written.
+// A linear kernel that follows on the stream may start early and fetch planes before it waits for
+// its predecessor; with this launch in between, that predecessor is the fence, and the fence did
+// not start before the split kernel had finished and its writes were visible.
+__global__ void plane_fence_kernel() {}
+
 }  // namespace
 
 cudaError_t launch_magnitude_stat(const uint16_t* w, int64_t n, unsigned* stat, cudaStream_t stream) {
@@ -98,6 +104,8 @@ cudaError_t launch_split(const uint16_t* w, uint8_t* p, uint8_t* r, int64_t n, i
         split_kernel<kEncE5M2><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint4*>(w),
                                                                reinterpret_cast<uint4*>(p),
                                                                reinterpret_cast<uint4*>(r), n16);
+    count_launch();
+    plane_fence_kernel<<<1, 32, 0, stream>>>();
     count_launch();
     return cudaGetLastError();
 }

@@ -317,24 +317,49 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         // Stages are filled two at a time when the ring is deep enough: the two boxes cover 256
         // adjacent bytes of every weight row, which DRAM serves noticeably better than 128.
         const bool pair = (num_stages >= 6) && (num_stages % 2 == 0);
-        // While the preceding kernel drains, pull this CTA's first plane tiles into L2.  L2 is the
-        // point of coherence, so this is safe even if that kernel is still writing the planes; the
-        // loads proper are issued only after the dependency wait.
-        // (A rolling L2 prefetch further ahead during the main loop was measured slower.)
-        const int l2_ahead = 2 * num_stages;
-        if (elect_one()) {
-            const int ahead = num_kb < l2_ahead ? num_kb : l2_ahead;
-            for (int i = 0; i < ahead; ++i) {
+        // First pass over the ring.  The planes are model state: (dense launches) their loads are
+        // issued BEFORE the dependency wait, so that the ring fills while the preceding kernel
+        // drains; only the activations -- that kernel's output in a decoder -- wait for it.  A
+        // stage's barrier expects the bytes of both, so it completes when the later one lands.
+        const int first = num_kb < num_stages ? num_kb : num_stages;
+        auto load_planes = [&](int i, int s) {
+            const uint32_t full = smem_u32(&bar_full[s]);
+            const uint32_t dst = smem_base + (uint32_t)s * kStage;
+            const int k = (rank + i * split) * kBlockK;
+            mbar_arrive_expect_tx(full, (uint32_t)kStage);
+            tma_load_2d(dst, &map_p, full, k, plane_row0);
+            if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, plane_row0);
+        };
+        auto load_x = [&](int i, int s) {
+            const uint32_t full = smem_u32(&bar_full[s]);
+            const uint32_t dst = smem_base + (uint32_t)s * kStage;
+            const int k = (rank + i * split) * kBlockK;
+#pragma unroll
+            for (int t = 0; t < kXAtoms; ++t)
+                tma_load_2d(dst + kXOffset + (uint32_t)(t * TN * 128), &map_x, full, k + t * 64, m0);
+        };
+        if (!GROUPED && elect_one()) {
+            for (int i = 0; i < first; ++i) load_planes(i, i);
+            // ... and the plane tiles of the second pass are pulled into L2 meanwhile.
+            // (A rolling L2 prefetch further ahead during the main loop was measured slower.)
+            const int ahead = num_kb < 2 * num_stages ? num_kb : 2 * num_stages;
+            for (int i = first; i < ahead; ++i) {
                 const int k = (rank + i * split) * kBlockK;
                 tma_prefetch_l2_2d(&map_p, k, plane_row0);
                 if (FULL) tma_prefetch_l2_2d(&map_r, k, plane_row0);
             }
         }
         __syncwarp();
-        grid_dependency_wait();  // everything read from global memory may come from the preceding kernel
-        int s = 0;
-        uint32_t ph = 0;
-        for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
+        if (!GROUPED) grid_dependency_wait();   // grouped launches waited before reading the tile list
+        if (elect_one())
+            for (int i = 0; i < first; ++i) {
+                if (GROUPED) load_planes(i, i);
+                load_x(i, i);
+            }
+        __syncwarp();
+        int s = first == num_stages ? 0 : first;
+        uint32_t ph = first == num_stages ? 1u : 0u;
+        for (int i = first; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
             if (!pair || (i & 1) == 0) {
                 ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);
                 if (ok && pair && i + 1 < num_kb) {     // pairs never wrap: the ring depth is even
@@ -345,15 +370,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             if (!ok) break;
             DPS_STAMP(0, i);
             if (elect_one()) {
-                const uint32_t full = smem_u32(&bar_full[s]);
-                const uint32_t dst = smem_base + (uint32_t)s * kStage;
-                const int k = (rank + i * split) * kBlockK;
-                mbar_arrive_expect_tx(full, (uint32_t)kStage);
-                tma_load_2d(dst, &map_p, full, k, plane_row0);
-                if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, plane_row0);
-#pragma unroll
-                for (int t = 0; t < kXAtoms; ++t)
-                    tma_load_2d(dst + kXOffset + (uint32_t)(t * TN * 128), &map_x, full, k + t * 64, m0);
+                load_planes(i, s);
+                load_x(i, s);
             }
             __syncwarp();
         }
