@@ -206,6 +206,12 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
 // read correctly afterwards.
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
+// Barrier among `threads` threads of the CTA (a multiple of 32) on hardware barrier `id` (1-15;
+// 0 is __syncthreads).
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 __device__ __forceinline__ void grid_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }

@@ -47,7 +47,11 @@ constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
 #ifndef DPS_BK64_FROM
 #define DPS_BK64_FROM 96
 #endif
-__host__ __device__ constexpr int block_k(bool full, int tn) {
+#ifndef DPS_RB2_FAST_BK
+#define DPS_RB2_FAST_BK 128
+#endif
+__host__ __device__ constexpr int block_k(bool full, int tn, int rb = 1) {
+    if (rb == 2) return full ? 64 : DPS_RB2_FAST_BK;
     return (tn >= DPS_BK64_FROM || (full && tn <= 64)) ? 64 : 128;
 }
 constexpr int kMaxAStages = 4;   // barrier array size for the A ring in tensor memory
@@ -59,9 +63,11 @@ __host__ __device__ constexpr int cta_threads(bool full, int tn) { return 64 + z
 constexpr int kMaxStages = 12;
 constexpr int kMaxSplit = 8;     // portable cluster size
 
-__host__ __device__ constexpr int plane_stage_bytes(bool full, int tn) { return kTileRows * block_k(full, tn); }
-__host__ __device__ constexpr int stage_bytes(bool full, int tn) {
-    return plane_stage_bytes(full, tn) * (full ? 2 : 1) + tn * block_k(full, tn) * 2;
+__host__ __device__ constexpr int plane_stage_bytes(bool full, int tn, int rb = 1) {
+    return rb * kTileRows * block_k(full, tn, rb);
+}
+__host__ __device__ constexpr int stage_bytes(bool full, int tn, int rb = 1) {
+    return plane_stage_bytes(full, tn, rb) * (full ? 2 : 1) + tn * block_k(full, tn, rb) * 2;
 }
 // Columns to allocate: accumulator + A ring.  Tiles of up to 64 tokens leave room for three A
 // slots inside 256 columns (two CTAs per SM); wider tiles keep two.
@@ -70,8 +76,10 @@ __host__ __device__ constexpr int a_slots(bool full, int tn) { return block_k(fu
 __host__ __device__ constexpr int a_slots_max(bool full, int tn) {
     return (tn <= 64 && a_slots(full, tn) < 3) ? 3 : a_slots(full, tn);
 }
-__host__ __device__ constexpr int tmem_cols(bool full, int tn) {
-    int need = tn + a_slots_max(full, tn) * (block_k(full, tn) / 2);
+// Two row blocks: two accumulators, and each zip group owns two A slots of its own.
+__host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
+    int need = rb == 2 ? 2 * tn + 4 * (block_k(full, tn, rb) / 2)
+                       : tn + a_slots_max(full, tn) * (block_k(full, tn) / 2);
     int c = 32;
     while (c < need) c <<= 1;
     return c;
@@ -82,11 +90,17 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn) {
 #ifdef DPS_TRACE
 constexpr int kTraceBlocks = 64, kTraceEvents = 16;
 __device__ long long g_trace[kTraceBlocks * kTraceEvents];
-__device__ unsigned long long g_cta_times[2048 * 8];
+__device__ unsigned long long g_cta_times[2 * 2048 * 12];
 #define DPS_CTA_STAMP(ev)                                                                          \
     do {                                                                                           \
         const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);           \
-        if (threadIdx.x == 64 && cta_ < 2048) g_cta_times[cta_ * 8 + (ev)] = global_timer_ns();    \
+        if (threadIdx.x == 64 && cta_ < 2048) g_cta_times[(prm.trace_slot * 2048 + cta_) * 12 + (ev)] = global_timer_ns(); \
+    } while (0)
+#define DPS_CTA_STAMP_T(ev, tid)                                                                   \
+    do {                                                                                           \
+        const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);           \
+        if (threadIdx.x == (tid) && cta_ < 2048)                                                   \
+            g_cta_times[(prm.trace_slot * 2048 + cta_) * 12 + (ev)] = global_timer_ns();           \
     } while (0)
 #ifdef DPS_TRACE_BLOCKS
 #define DPS_STAMP(ev, i)                                                                          \
@@ -101,6 +115,7 @@ __device__ unsigned long long g_cta_times[2048 * 8];
 #else
 #define DPS_STAMP(ev, i) do { } while (0)
 #define DPS_CTA_STAMP(ev) do { } while (0)
+#define DPS_CTA_STAMP_T(ev, tid) do { } while (0)
 #endif
 
 // Grouped (MoE) launches: blockIdx.y indexes a list of token tiles built on the device by the
@@ -119,7 +134,9 @@ struct UmmaParams {
     int split;       // K split = cluster size along z; partial tiles are summed through DSMEM
     int red_offset;  // byte offset (from the aligned base of dynamic smem) of the split-K mailbox
     int* status;
-
+#ifdef DPS_TRACE
+    int trace_slot;  // which half of the CTA time table this launch writes
+#endif
 };
 
 // What a zip warp needs to know about its CTA's pipeline.
@@ -133,11 +150,14 @@ struct ZipCtx {
 // Zip loop of one warp: for each of its K blocks, wait for the planes to land and for the A slot
 // to be free, rebuild 128 FP16 weights of this thread's row from the plane bytes and store them
 // into tensor memory.  Returns false if a wait timed out.
-template <int ENC, bool FULL, int TN>
+//
+// RB == 2: the stage holds two row blocks (256 plane rows) that share one activation tile; zip
+// group g rebuilds row block g of EVERY K block into its own two A slots (2g, 2g + 1).
+template <int ENC, bool FULL, int TN, int RB>
 __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
-    constexpr int kBlockK = block_k(FULL, TN);
+    constexpr int kBlockK = block_k(FULL, TN, RB);
     constexpr int kACols = kBlockK / 2;
-    constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN);
+    constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
     constexpr int kSlots = a_slots(FULL, TN);
     bool ok = true;
     // Ring positions are advanced incrementally (no division in the loop).  Every stage and every A
@@ -147,10 +167,11 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
     int s = 0;
     uint32_t s_parity = 0;   // phase parity of stage s
     for (int i = 0; i < z.num_kb && ok; ++i, s = (s + 1 == z.num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
-        const int a = z.slot_per_stage ? s : (i & (kSlots - 1));
+        const int a = RB == 2 ? 2 * z.group + (i & 1) : z.slot_per_stage ? s : (i & (kSlots - 1));
         const int owner = z.slot_per_stage ? (s & 1) : (i & (zip_groups(FULL, TN) - 1));
-        if (owner != z.group) continue;
-        const uint32_t a_parity = z.slot_per_stage ? s_parity : (uint32_t)(i / kSlots) & 1u;
+        if (RB == 1 && owner != z.group) continue;
+        const uint32_t a_parity = RB == 2 ? (uint32_t)(i >> 1) & 1u
+                                          : z.slot_per_stage ? s_parity : (uint32_t)(i / kSlots) & 1u;
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(4, i);
         ok = mbar_wait(smem_u32(&z.bar_full[s]), s_parity);
         ok = __all_sync(0xFFFFFFFFu, ok);
@@ -158,7 +179,8 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(5, i);
         // Read and rebuild the weights FIRST, into registers: that needs the stage, not the A slot,
         // so it overlaps the MMAs that are still reading the slot's previous contents.
-        const uint32_t prow = z.smem_base + (uint32_t)s * z.stage_bytes + (uint32_t)z.row * kBlockK;
+        const uint32_t prow = z.smem_base + (uint32_t)s * z.stage_bytes +
+                              (uint32_t)((RB == 2 ? z.group * kTileRows : 0) + z.row) * kBlockK;
         uint32_t h[kACols];
 #pragma unroll
         for (int c = 0; c < kBlockK / 16; ++c) {
@@ -203,19 +225,24 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
 }
 
 // ENC == 0 (grouped launches only): the encoding is a per-expert run-time value.
-template <int ENC, bool FULL, int TN, bool GROUPED>
-__global__ void __launch_bounds__(cta_threads(FULL, TN), (tmem_cols(FULL, TN) <= 256 ? 2 : 1))
+// RB = row blocks of 128 weight rows per CTA.  With RB == 2 one activation tile per stage feeds two
+// accumulators, which halves the activation bytes an SM pulls out of L2 per weight byte -- the
+// limit of the grouped (MoE) launches, whose token tiles are wide but whose planes are read once.
+// RB == 2 supports neither a K split nor the odd ring; each zip group serves one row block.
+template <int ENC, bool FULL, int TN, bool GROUPED, int RB = 1>
+__global__ void __launch_bounds__(cta_threads(FULL, TN), (tmem_cols(FULL, TN, RB) <= 256 ? 2 : 1))
 umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
                    const __grid_constant__ CUtensorMap map_x, const UmmaParams prm, const GroupedParams gp) {
-    constexpr int kBlockK = block_k(FULL, TN);
+    constexpr int kBlockK = block_k(FULL, TN, RB);
     constexpr int kXAtoms = kBlockK / 64;    // the x tile is stored as 64-element (128-byte) swizzle atoms
     constexpr int kACols = kBlockK / 2;      // TMEM columns of one A slot (two FP16 per column)
-    constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN);
+    constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
     constexpr int kSlots = a_slots(FULL, TN);
-    constexpr int kStage = stage_bytes(FULL, TN);
+    constexpr int kStage = stage_bytes(FULL, TN, RB);
     constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
-    constexpr uint32_t kCols = tmem_cols(FULL, TN);
-    constexpr uint32_t kIdesc = umma_idesc_f16(kTileRows, TN);
+    constexpr uint32_t kCols = tmem_cols(FULL, TN, RB);
+    static_assert(RB == 1 || RB == 2, "one or two row blocks per CTA");
+    static_assert(RB == 1 || zip_groups(FULL, TN) == 2, "two row blocks need exactly two zip groups");
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[kMaxStages];
@@ -232,7 +259,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         unsigned smid_;
         asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_));
         const int cta_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-        if (threadIdx.x == 64 && cta_ < 2048) g_cta_times[cta_ * 8 + 5] = smid_;
+        if (threadIdx.x == 64 && cta_ < 2048) g_cta_times[(prm.trace_slot * 2048 + cta_) * 12 + 5] = smid_;
     }
 #endif
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -240,7 +267,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const int num_stages = prm.num_stages;
     constexpr int kZipGroups = zip_groups(FULL, TN);
     constexpr int kThreads = cta_threads(FULL, TN);
-    const bool slot_per_stage = (num_stages % kZipGroups) != 0;   // only the 3-deep ring
+    const bool slot_per_stage = RB == 1 && (num_stages % kZipGroups) != 0;   // only the 3-deep ring
     // Tile order (dense launches with several token tiles): CTAs are handed out x-fastest, so walk
     // groups of 8 row tiles x all token tiles.  The CTAs running at any moment then share 8 row
     // tiles of planes and a few dozen activation tiles, which stay in L2, instead of sweeping
@@ -256,7 +283,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         row_tile = group * kRowGroup + within % rows_here;
         tok_tile = within / rows_here;
     }
-    const int n0 = row_tile * kTileRows;
+    const int n0 = row_tile * kTileRows * RB;
     int m0 = tok_tile * TN;          // first token (dense) / first sorted row (grouped) of the tile
     int tile_tokens = TN;            // valid token columns of the tile (grouped)
     int plane_row0 = n0;             // first plane row of the tile in the [E * N][K] view
@@ -270,6 +297,11 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         plane_row0 = t.x * prm.N + n0;
         e5m2 = (gp.e5m2[t.x >> 5] >> (t.x & 31)) & 1u;
     }
+    // UMMA N of this tile.  A grouped tile multiplies only the token columns it has (rounded up to
+    // 16): at 64-96 tokens per expert a fast-mode MoE layer sits at the ridge between HBM and the
+    // tensor pipe, and padded columns are tensor time.  The activation box still brings TN rows.
+    const int mma_n = GROUPED ? min(TN, (tile_tokens + 15) & ~15) : TN;
+    const uint32_t idesc = umma_idesc_f16(kTileRows, mma_n);
     const int total_kb = (prm.K + kBlockK - 1) / kBlockK;
     const int split = prm.split;
     const int rank = (split > 1) ? (int)cluster_ctarank() : 0;   // == blockIdx.z
@@ -280,7 +312,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     if (threadIdx.x == 0) {
         for (int s = 0; s < num_stages; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_empty[s]), 5);  // 4 zip warps + 1 tcgen05.commit
+            mbar_init(smem_u32(&bar_empty[s]), RB == 2 ? 9 : 5);  // 4 zip warps per reader group + 1 tcgen05.commit
         }
         for (int a = 0; a < kMaxAStages; ++a) {
             mbar_init(smem_u32(&bar_a_full[a]), 4);
@@ -298,8 +330,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     tc_fence_after_sync();
     DPS_CTA_STAMP(1);
     const uint32_t tmem_base = tmem_base_slot;
-    const uint32_t tmem_d = tmem_base;           // TN accumulator columns
-    const uint32_t tmem_a = tmem_base + TN;      // A ring: slots of kACols columns of packed FP16 pairs
+    const uint32_t tmem_d = tmem_base;           // TN accumulator columns per row block
+    const uint32_t tmem_a = tmem_base + RB * TN; // A ring: slots of kACols columns of packed FP16 pairs
 
     // Split-K sums.  TN <= 64 ("push"): every CTA owns the tokens c with c % split == rank and has a
     // mailbox mail[source rank][slot = c / split][row] in its own shared memory, outside the stage
@@ -350,7 +382,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             }
         }
         __syncwarp();
+        DPS_CTA_STAMP_T(8, 0);
         if (!GROUPED) grid_dependency_wait();   // grouped launches waited before reading the tile list
+        DPS_CTA_STAMP_T(9, 0);
         if (elect_one())
             for (int i = 0; i < first; ++i) {
                 if (GROUPED) load_planes(i, i);
@@ -380,6 +414,37 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         int s = 0;
         uint32_t s_parity = 0;
         for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
+            const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
+            if (RB == 2) {
+                // row block g: A slot 2g + (i & 1) of zip group g, accumulator columns [g * TN, (g + 1) * TN)
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    const int a = 2 * g + (i & 1);
+                    if (g == 0) DPS_STAMP(1, i);
+                    ok = mbar_wait(smem_u32(&bar_a_full[a]), (uint32_t)(i >> 1) & 1u);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    if (g == 0) DPS_STAMP(2, i);
+                    tc_fence_after_sync();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int j = 0; j < kBlockK / 16; ++j) {
+                            const uint64_t bdesc = umma_desc_k_sw128(xbase + (uint32_t)((j >> 2) * TN * 128)) +
+                                                   (uint64_t)((j & 3) * 2);
+                            umma_f16_ts(tmem_d + (uint32_t)(g * TN), tmem_a + (uint32_t)(a * kACols + j * 8), bdesc,
+                                        idesc, (i > 0 || j > 0) ? 1u : 0u);
+                        }
+                        umma_commit(smem_u32(&bar_a_empty[a]));
+                        if (g == 1) {
+                            umma_commit(smem_u32(&bar_empty[s]));
+                            if (i == num_kb - 1) umma_commit(smem_u32(&bar_d_full));
+                        }
+                    }
+                    __syncwarp();
+                }
+                DPS_STAMP(3, i);
+                continue;
+            }
             const int a = slot_per_stage ? s : (i & (kSlots - 1));
             const uint32_t pair_parity = (uint32_t)(i / kSlots) & 1u;
             // The zip warps waited for this stage's TMA loads before they arrived on a_full, so the
@@ -389,15 +454,15 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             DPS_STAMP(2, i);
+            if (i == 0) DPS_CTA_STAMP_T(10, 32);
             tc_fence_after_sync();
             if (elect_one()) {
-                const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
 #pragma unroll
                 for (int j = 0; j < kBlockK / 16; ++j) {
                     // 16 K elements = 32 bytes inside the 128-byte swizzle atom (j / 4)
                     const uint64_t bdesc = umma_desc_k_sw128(xbase + (uint32_t)((j >> 2) * TN * 128)) +
                                            (uint64_t)((j & 3) * 2);
-                    umma_f16_ts(tmem_d, tmem_a + (uint32_t)(a * kACols + j * 8), bdesc, kIdesc,
+                    umma_f16_ts(tmem_d, tmem_a + (uint32_t)(a * kACols + j * 8), bdesc, idesc,
                                 (i > 0 || j > 0) ? 1u : 0u);
                 }
                 umma_commit(smem_u32(&bar_empty[s]));
@@ -424,55 +489,93 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
         if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2)) {
             // encoding known only at run time (one per expert): uniform branch per CTA
-            ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN>(zc) : zip_blocks<kEncE4M3, FULL, TN>(zc);
+            ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc);
         } else {
-            ok = zip_blocks<ENC, FULL, TN>(zc);
+            ok = zip_blocks<ENC, FULL, TN, RB>(zc);
         }
-        // epilogue (first zip group): D[row][token] -> y[token][n0 + row], or -> red for split K
-        if (group == 0) {
-            // E4M3 fast mode multiplied with 2^8 times the weights (hardware FP8 conversion)
-            const float out_scale = (!FULL && !e5m2) ? 0.00390625f : 1.0f;
+        // E4M3 fast mode multiplied with 2^8 times the weights (hardware FP8 conversion)
+        const float out_scale = (!FULL && !e5m2) ? 0.00390625f : 1.0f;
+        if (split == 1) {
+            // ---- epilogue without a K split: D -> FP16 -> shared memory -> y, by all zip warps ----
+            // The accumulator is drained into a [token][row] FP16 tile that overlays the idle stage
+            // ring (every load has been consumed once the last MMA is complete), and then written
+            // out with 16-byte stores: one warp instruction covers 512 contiguous bytes of a row
+            // of y.  Storing straight from the accumulator registers (2 bytes per thread per
+            // token, 64 bytes per warp instruction) took 5 us per 256 x 96 tile, with nothing
+            // else running on the SM.
+            constexpr int kRowsCta = kTileRows * RB;
+            constexpr int kColsPerGroup = (RB == 2 || TN < 32) ? TN : TN / 2;   // RB == 1: the groups share the columns
+            const int ncols = GROUPED ? tile_tokens : min(TN, prm.M - m0);     // token columns that exist
+            if (ok) ok = mbar_wait(smem_u32(&bar_d_full), 0u);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            DPS_CTA_STAMP(2);
+            const bool drains = RB == 2 || TN >= 32 || group == 0;
+            if (ok && drains) {
+                tc_fence_after_sync();
+                const int rb = RB == 2 ? group : 0;
+                const int cbeg = (RB == 1 && TN >= 32) ? group * kColsPerGroup : 0;
+#pragma unroll
+                for (int cc = 0; cc < kColsPerGroup; cc += 16) {
+                    const int c0 = cbeg + cc;
+                    if (c0 >= ncols) break;                       // warp-uniform
+                    uint32_t v[16];
+                    tmem_ld_32x32b_x16(tmem_d + lane_base + (uint32_t)(rb * TN + c0), v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const __half h = __float2half_rn(__uint_as_float(v[j]) * out_scale);
+                        const uint32_t addr = smem_base + (uint32_t)(((c0 + j) * kRowsCta + rb * kTileRows + row) * 2);
+                        asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(h)) : "memory");
+                    }
+                }
+            }
+            named_barrier_sync(1, kZipGroups * 128);              // the zip warps only
+            DPS_CTA_STAMP(3);
+            if (ok) {
+                constexpr int kChunks = kRowsCta / 8;             // 16-byte pieces of one token's rows
+                const int zt = (int)threadIdx.x - 64;             // index among the zip threads
+                for (int item = zt; item < ncols * kChunks; item += kZipGroups * 128) {
+                    const int c = item / kChunks, q = item % kChunks;
+                    const int n = n0 + q * 8;
+                    if (n >= prm.N) continue;                     // N is a multiple of 8: a piece is in or out
+                    const int m = GROUPED ? gp.sorted_rows[m0 + c] : m0 + c;
+                    uint4 val;
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                                 : "r"(smem_base + (uint32_t)((c * kRowsCta + q * 8) * 2)));
+                    *reinterpret_cast<uint4*>(prm.y + (int64_t)m * prm.N + n) = val;
+                }
+            }
+        } else if (group == 0) {
+            // ---- epilogue with a K split (first zip group): partial sums -> mailbox / red ----
             if (ok) ok = mbar_wait(smem_u32(&bar_d_full), 0u);
             ok = __all_sync(0xFFFFFFFFu, ok);
             DPS_CTA_STAMP(2);
             if (ok) {
                 tc_fence_after_sync();
-                const int n = n0 + row;
 #pragma unroll
                 for (int c0 = 0; c0 < TN; c0 += 16) {
                     uint32_t v[16];
                     tmem_ld_32x32b_x16(tmem_d + lane_base + (uint32_t)c0, v);
                     tmem_wait_ld();
-                    if (split > 1 && kPush) {
+                    if (kPush) {
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const int c = c0 + j, owner = c % split, slot = c / split;
                             const uint32_t local = mail_addr + (uint32_t)(((rank * slots + slot) * kTileRows + row) * 4);
                             st_cluster_f32(map_to_cta(local, (uint32_t)owner), __uint_as_float(v[j]) * out_scale);
                         }
-                    } else if (split > 1) {
+                    } else {
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
                             red[(c0 + j) * kTileRows + row] = __uint_as_float(v[j]) * out_scale;
-                    } else if (n < prm.N) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            int m = m0 + c0 + j;
-                            bool valid = m < prm.M;
-                            if (GROUPED) {
-                                valid = (c0 + j) < tile_tokens;
-                                if (valid) m = gp.sorted_rows[m];
-                            }
-                            if (valid)
-                                prm.y[(int64_t)m * prm.N + n] = __float2half_rn(__uint_as_float(v[j]) * out_scale);
-                        }
                     }
                 }
             }
         }
     }
     if (!ok) atomicExch(prm.status, (int)DPS_ERR_CUDA);
-    DPS_CTA_STAMP(3);
+    if (split > 1) DPS_CTA_STAMP(3);
 
     if (split > 1 && kPush) {
         __syncthreads();
@@ -682,6 +785,10 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     prm.split = split;
     prm.red_offset = stages * kStage;
     prm.status = status;
+#ifdef DPS_TRACE
+    static int trace_launches = 0;
+    prm.trace_slot = (trace_launches++) & 1;
+#endif
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)row_tiles, (unsigned)tok_tiles, (unsigned)split);
@@ -732,28 +839,29 @@ extern "C" __attribute__((visibility("default"))) int dps_debug_trace(long long*
     return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * n);
 }
 extern "C" __attribute__((visibility("default"))) int dps_debug_cta_times(unsigned long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, g_cta_times, sizeof(unsigned long long) * 2048 * 8);
+    return (int)cudaMemcpyFromSymbol(out, g_cta_times, sizeof(unsigned long long) * 2 * 2048 * 12);
 }
 #endif
 
 namespace {
 
-template <bool FULL, int TN>
+template <bool FULL, int TN, int RB>
 cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, const uint8_t* p, const uint8_t* r,
                               void* y, int64_t A, int64_t N, int64_t K, int32_t E, const void* tiles,
                               const int32_t* num_tiles, const int32_t* sorted_rows, int max_tiles, int* status,
                               cudaStream_t stream) {
-    constexpr int kStage = stage_bytes(FULL, TN);
+    constexpr int kStage = stage_bytes(FULL, TN, RB);
     constexpr int kZipGroups = zip_groups(FULL, TN);
     constexpr int kThreads = cta_threads(FULL, TN);
-    constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
+    constexpr int kCtasPerSm = tmem_cols(FULL, TN, RB) <= 256 ? 2 : 1;
     constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
     int stages = kSmemTotal / kStage;
     if (stages > 8) stages = 8;
     if (stages < 2) stages = 2;
-    stages -= stages % kZipGroups;
+    if (RB == 1) stages -= stages % kZipGroups;   // stages alternate between the zip groups
+    else if (stages >= 6) stages &= ~1;           // any depth works; even ones fill two stages at a time
     const size_t smem = (size_t)stages * kStage + 1024;
-    auto kernel = umma_linear_kernel<0, FULL, TN, true>;
+    auto kernel = umma_linear_kernel<0, FULL, TN, true, RB>;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
@@ -764,13 +872,13 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
         configured = true;
     }
     CUtensorMap mp, mr, mx;
-    constexpr int kBlockK = block_k(FULL, TN);
+    constexpr int kBlockK = block_k(FULL, TN, RB);
     constexpr CUtensorMapSwizzle kPlaneSwizzle = kBlockK == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
-    if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows,
+    if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows * RB,
                      kBlockK, kPlaneSwizzle))
         return cudaErrorInvalidValue;
     if (FULL) {
-        if (!make_map_2d(&mr, r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows,
+        if (!make_map_2d(&mr, r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)E * (uint64_t)N, (uint64_t)K, kTileRows * RB,
                          kBlockK, kPlaneSwizzle))
             return cudaErrorInvalidValue;
     } else {
@@ -779,7 +887,7 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     if (!make_map_2d(&mx, x_sorted, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)A, (uint64_t)K, TN, 64,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return cudaErrorInvalidValue;
-    UmmaParams prm;
+    UmmaParams prm = {};
     prm.y = static_cast<__half*>(y);
     prm.M = (int)A;
     prm.N = (int)N;
@@ -795,7 +903,7 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     for (int i = 0; i < 32; ++i) gp.e5m2[i] = e5m2_mask[i];
 
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((N + kTileRows - 1) / kTileRows), (unsigned)max_tiles, 1);
+    cfg.gridDim = dim3((unsigned)((N + kTileRows * RB - 1) / (kTileRows * RB)), (unsigned)max_tiles, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -825,19 +933,35 @@ cudaError_t launch_umma_grouped(int mode, const uint32_t* e5m2_mask, const void*
                                 const uint8_t* r, void* y, int64_t A, int64_t N, int64_t K, int32_t E, int tn,
                                 const void* tiles, const int32_t* num_tiles, const int32_t* sorted_rows,
                                 int max_tiles, int* status, cudaStream_t stream) {
+    // Two row blocks per CTA for wide token tiles, when that still leaves every SM a CTA: the
+    // activation tile is then fetched from L2 once per 256 weight rows instead of once per 128.
+    // DPS_GROUPED_RB=1|2 overrides (tuning knob).
+    static const int rb_forced = [] {
+        const char* e = getenv("DPS_GROUPED_RB");
+        return e ? atoi(e) : 0;
+    }();
+    const bool two = rb_forced ? rb_forced == 2
+                               : (tn >= 64 && ((N + 2 * kTileRows - 1) / (2 * kTileRows)) * max_tiles >= sm_count());
+#define DPS_GROUPED_CALL(FULLV, TNV, RBV)                                                                         \
+    launch_grouped_tn<FULLV, TNV, RBV>(e5m2_mask, x_sorted, p, r, y, A, N, K, E, tiles, num_tiles, sorted_rows,  \
+                                       max_tiles, status, stream)
 #define DPS_GROUPED_CASE(TNV)                                                                                     \
     if (tn == TNV)                                                                                                \
-        return mode == DPS_MODE_FULL                                                                              \
-                   ? launch_grouped_tn<true, TNV>(e5m2_mask, x_sorted, p, r, y, A, N, K, E, tiles, num_tiles,     \
-                                                  sorted_rows, max_tiles, status, stream)                        \
-                   : launch_grouped_tn<false, TNV>(e5m2_mask, x_sorted, p, r, y, A, N, K, E, tiles, num_tiles,    \
-                                                   sorted_rows, max_tiles, status, stream);
+        return mode == DPS_MODE_FULL ? DPS_GROUPED_CALL(true, TNV, 1) : DPS_GROUPED_CALL(false, TNV, 1);
+#define DPS_GROUPED_CASE2(TNV)                                                                                    \
+    if (tn == TNV && two)                                                                                         \
+        return mode == DPS_MODE_FULL ? DPS_GROUPED_CALL(true, TNV, 2) : DPS_GROUPED_CALL(false, TNV, 2);
+    DPS_GROUPED_CASE2(64)
+    DPS_GROUPED_CASE2(96)
+    DPS_GROUPED_CASE2(128)
     DPS_GROUPED_CASE(16)
     DPS_GROUPED_CASE(32)
     DPS_GROUPED_CASE(64)
     DPS_GROUPED_CASE(96)
     DPS_GROUPED_CASE(128)
 #undef DPS_GROUPED_CASE
+#undef DPS_GROUPED_CASE2
+#undef DPS_GROUPED_CALL
     return cudaErrorInvalidValue;
 }
 
