@@ -139,6 +139,12 @@ struct UmmaParams {
 #endif
 };
 
+// Two floats -> packed FP16 pair (first in the low half), round to nearest even.
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+
 // What a zip warp needs to know about its CTA's pipeline.
 struct ZipCtx {
     int group, warp, lane, row, num_kb, num_stages, stage_bytes;
@@ -546,15 +552,18 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                     *reinterpret_cast<uint4*>(prm.y + (int64_t)m * prm.N + n) = val;
                 }
             }
-        } else if (group == 0) {
-            // ---- epilogue with a K split (first zip group): partial sums -> mailbox / red ----
+        } else if (group == 0 || TN >= 32) {
+            // ---- epilogue with a K split: partial sums -> mailbox / red; the zip groups share the columns ----
+            constexpr int kColsPerGroup = TN >= 32 ? TN / 2 : TN;
+            const int cbeg = TN >= 32 ? group * kColsPerGroup : 0;
             if (ok) ok = mbar_wait(smem_u32(&bar_d_full), 0u);
             ok = __all_sync(0xFFFFFFFFu, ok);
             DPS_CTA_STAMP(2);
             if (ok) {
                 tc_fence_after_sync();
 #pragma unroll
-                for (int c0 = 0; c0 < TN; c0 += 16) {
+                for (int cc = 0; cc < kColsPerGroup; cc += 16) {
+                    const int c0 = cbeg + cc;
                     uint32_t v[16];
                     tmem_ld_32x32b_x16(tmem_d + lane_base + (uint32_t)c0, v);
                     tmem_wait_ld();
@@ -582,14 +591,25 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         cluster_sync_all();  // release/acquire: every peer's stores into this CTA's mailbox are visible
         DPS_CTA_STAMP(4);
         const float* mail = reinterpret_cast<const float*>(smem_raw + (smem_base - smem_u32(smem_raw)) + prm.red_offset);
-        for (int e = threadIdx.x; e < slots * kTileRows; e += kThreads) {
-            const int slot = e / kTileRows, r = e % kTileRows;
+        // one item = 8 consecutive rows of one owned token: 16 bytes of y
+        for (int e = threadIdx.x; e < slots * (kTileRows / 8); e += kThreads) {
+            const int slot = e / (kTileRows / 8), r = (e % (kTileRows / 8)) * 8;
             const int c = slot * split + rank;
             const int m = m0 + c, n = n0 + r;
-            if (c >= TN || m >= prm.M || n >= prm.N) continue;
-            float acc = 0.f;
-            for (int j = 0; j < split; ++j) acc += mail[(j * slots + slot) * kTileRows + r];
-            prm.y[(int64_t)m * prm.N + n] = __float2half_rn(acc);
+            if (c >= TN || m >= prm.M || n >= prm.N) continue;   // N is a multiple of 8
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int j = 0; j < split; ++j) {
+                const float4* src = reinterpret_cast<const float4*>(mail + (j * slots + slot) * kTileRows + r);
+                const float4 a = src[0], b = src[1];
+                acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+                acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
+            }
+            uint4 out;
+            out.x = pack_half2(acc[0], acc[1]);
+            out.y = pack_half2(acc[2], acc[3]);
+            out.z = pack_half2(acc[4], acc[5]);
+            out.w = pack_half2(acc[6], acc[7]);
+            *reinterpret_cast<uint4*>(prm.y + (int64_t)m * prm.N + n) = out;
         }
     } else if (split > 1) {
         __syncthreads();
@@ -812,6 +832,72 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     return e;
 }
 
+// Dense launch with two row blocks per CTA (256 weight rows share each activation tile): no K
+// split, one CTA per SM unless the tile is narrow.
+template <int ENC, bool FULL, int TN>
+cudaError_t launch_tn_rb2(const void* x, const uint8_t* p, const uint8_t* r, void* y, int64_t M, int64_t N, int64_t K,
+                          int* status, cudaStream_t stream) {
+    constexpr int kRb = 2;
+    constexpr int kStage = stage_bytes(FULL, TN, kRb);
+    constexpr int kThreads = cta_threads(FULL, TN);
+    constexpr int kCtasPerSm = tmem_cols(FULL, TN, kRb) <= 256 ? 2 : 1;
+    constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
+    constexpr int kBlockK = block_k(FULL, TN, kRb);
+    constexpr CUtensorMapSwizzle kPlaneSwizzle = kBlockK == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    int stages = kSmemTotal / kStage;
+    if (stages > 8) stages = 8;
+    if (stages < 2) stages = 2;
+    if (stages >= 6) stages &= ~1;
+    const size_t smem = (size_t)stages * kStage + 1024;
+    auto kernel = umma_linear_kernel<ENC, FULL, TN, false, kRb>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    CUtensorMap mp, mr, mx;
+    if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, (uint64_t)K, kTileRows * kRb, kBlockK,
+                     kPlaneSwizzle))
+        return cudaErrorInvalidValue;
+    if (FULL) {
+        if (!make_map_2d(&mr, r, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, (uint64_t)K, kTileRows * kRb, kBlockK,
+                         kPlaneSwizzle))
+            return cudaErrorInvalidValue;
+    } else {
+        mr = mp;
+    }
+    if (!make_map_2d(&mx, x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)M, (uint64_t)K, TN, 64,
+                     CU_TENSOR_MAP_SWIZZLE_128B))
+        return cudaErrorInvalidValue;
+    UmmaParams prm = {};
+    prm.y = static_cast<__half*>(y);
+    prm.M = (int)M;
+    prm.N = (int)N;
+    prm.K = (int)K;
+    prm.num_stages = stages;
+    prm.split = 1;
+    prm.red_offset = 0;
+    prm.status = status;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((N + kTileRows * kRb - 1) / (kTileRows * kRb)), (unsigned)((M + TN - 1) / TN), 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    GroupedParams gp = {};
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, prm, gp);
+    count_launch();
+    return e;
+}
+
 template <int ENC, bool FULL>
 cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* y, int64_t M, int64_t N, int64_t K,
                        int* status, cudaStream_t stream) {
@@ -826,6 +912,18 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
         const char* e = getenv("DPS_FORCE_TN");
         return e ? atoi(e) : 0;
     }();
+    static const int rb_forced = [] {
+        const char* e = getenv("DPS_DENSE_RB");
+        return e ? atoi(e) : 0;
+    }();
+    // Fast mode with enough tiles to give every SM one and a half: 256 weight rows per CTA share
+    // each 128-token activation tile, which halves the activation bytes pulled out of L2 per
+    // FLOP (measured +2-8 % at 2048-8192 tokens; with fewer tiles the SMs run dry, and in full
+    // mode the zip warps would rebuild twice the weights per MMA cycle: -20 %).
+    // DPS_DENSE_RB=1|2 overrides (tuning knob).
+    const int64_t tiles_rb2 = ((N + 2 * kTileRows - 1) / (2 * kTileRows)) * ((M + 127) / 128);
+    const bool rb2 = rb_forced ? rb_forced == 2 : (!FULL && 2 * tiles_rb2 >= 3 * (int64_t)sm_count());
+    if (rb2 && M > 64) return launch_tn_rb2<ENC, FULL, 128>(x, p, r, y, M, N, K, status, stream);
     const bool wide = tn_forced ? tn_forced == 256 : (FULL ? M > 128 : (M > 128 && M <= 256));
     if (!wide) return launch_tn<ENC, FULL, 128>(x, p, r, y, M, N, K, status, stream);
     return launch_tn<ENC, FULL, 256>(x, p, r, y, M, N, K, status, stream);
