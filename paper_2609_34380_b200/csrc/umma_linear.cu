@@ -148,7 +148,6 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
 // What a zip warp needs to know about its CTA's pipeline.
 struct ZipCtx {
     int group, warp, lane, row, num_kb, num_stages, stage_bytes;
-    bool slot_per_stage;  // 3-deep ring: A slot = stage, owner group = stage % groups
     uint32_t smem_base, tmem_a, lane_base, sw;
     uint64_t *bar_full, *bar_empty, *bar_a_full, *bar_a_empty;
 };
@@ -164,20 +163,23 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
     constexpr int kBlockK = block_k(FULL, TN, RB);
     constexpr int kACols = kBlockK / 2;
     constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
-    constexpr int kSlots = a_slots(FULL, TN);
     bool ok = true;
     // Ring positions are advanced incrementally (no division in the loop).  Every stage and every A
     // slot always belongs to the same zip group, so that each waiter sees every phase of the barriers
-    // it waits on.  Even ring: blocks alternate between the groups and between two A slots.
-    // 3-deep ring: slot = stage, group = stage % groups.
+    // it waits on: stage s belongs to group s % 2 (any ring depth; with an even ring that is simply
+    // alternate K blocks), and group g owns the A slots g, g + 2, ... below the slot count, which
+    // it uses in turn.
+    constexpr int kTotalSlots = a_slots_max(FULL, TN);
+    const int my_slots = RB == 2 ? 2 : (kTotalSlots - z.group + 1) / 2;   // 1 or 2
     int s = 0;
     uint32_t s_parity = 0;   // phase parity of stage s
+    int cnt = 0;             // K blocks this group has rebuilt so far
     for (int i = 0; i < z.num_kb && ok; ++i, s = (s + 1 == z.num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
-        const int a = RB == 2 ? 2 * z.group + (i & 1) : z.slot_per_stage ? s : (i & (kSlots - 1));
-        const int owner = z.slot_per_stage ? (s & 1) : (i & (zip_groups(FULL, TN) - 1));
-        if (RB == 1 && owner != z.group) continue;
-        const uint32_t a_parity = RB == 2 ? (uint32_t)(i >> 1) & 1u
-                                          : z.slot_per_stage ? s_parity : (uint32_t)(i / kSlots) & 1u;
+        if (RB == 1 && (s & 1) != z.group) continue;
+        const int turn = my_slots == 2 ? (cnt & 1) : 0;
+        const int a = RB == 2 ? 2 * z.group + turn : z.group + 2 * turn;
+        const uint32_t a_parity = (uint32_t)(my_slots == 2 ? (cnt >> 1) : cnt) & 1u;
+        ++cnt;
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(4, i);
         ok = mbar_wait(smem_u32(&z.bar_full[s]), s_parity);
         ok = __all_sync(0xFFFFFFFFu, ok);
@@ -243,7 +245,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     constexpr int kXAtoms = kBlockK / 64;    // the x tile is stored as 64-element (128-byte) swizzle atoms
     constexpr int kACols = kBlockK / 2;      // TMEM columns of one A slot (two FP16 per column)
     constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
-    constexpr int kSlots = a_slots(FULL, TN);
     constexpr int kStage = stage_bytes(FULL, TN, RB);
     constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
     constexpr uint32_t kCols = tmem_cols(FULL, TN, RB);
@@ -273,7 +274,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     const int num_stages = prm.num_stages;
     constexpr int kZipGroups = zip_groups(FULL, TN);
     constexpr int kThreads = cta_threads(FULL, TN);
-    const bool slot_per_stage = RB == 1 && (num_stages % kZipGroups) != 0;   // only the 3-deep ring
     // Tile order (dense launches with several token tiles): CTAs are handed out x-fastest, so walk
     // groups of 8 row tiles x all token tiles.  The CTAs running at any moment then share 8 row
     // tiles of planes and a few dozen activation tiles, which stay in L2, instead of sweeping
@@ -417,8 +417,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (whole warp converged, one elected lane issues) ----------------
+        constexpr int kTotalSlots = a_slots_max(FULL, TN);
         int s = 0;
         uint32_t s_parity = 0;
+        int cnt[2] = {0, 0};     // K blocks taken from each zip group so far
         for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
             const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
             if (RB == 2) {
@@ -451,12 +453,17 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 DPS_STAMP(3, i);
                 continue;
             }
-            const int a = slot_per_stage ? s : (i & (kSlots - 1));
-            const uint32_t pair_parity = (uint32_t)(i / kSlots) & 1u;
+            // stage s belongs to zip group s % 2, which rotates through its own A slots (see zip_blocks)
+            const int g = s & 1;
+            const int g_slots = (kTotalSlots - g + 1) / 2;             // 1 or 2
+            const int turn = g_slots == 2 ? (cnt[g] & 1) : 0;
+            const int a = g + 2 * turn;
+            const uint32_t a_parity = (uint32_t)(g_slots == 2 ? (cnt[g] >> 1) : cnt[g]) & 1u;
+            ++cnt[g];
             // The zip warps waited for this stage's TMA loads before they arrived on a_full, so the
             // activation tile of the stage is complete and visible once a_full is: one wait, not two.
             DPS_STAMP(1, i);
-            ok = mbar_wait(smem_u32(&bar_a_full[a]), slot_per_stage ? s_parity : pair_parity);
+            ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             DPS_STAMP(2, i);
@@ -487,7 +494,6 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         ZipCtx zc;
         zc.group = group; zc.warp = warp; zc.lane = lane; zc.row = row;
         zc.num_kb = num_kb; zc.num_stages = num_stages; zc.stage_bytes = kStage;
-        zc.slot_per_stage = slot_per_stage;
         zc.smem_base = smem_base; zc.tmem_a = tmem_a; zc.lane_base = lane_base;
         // TMA swizzle of the plane tiles: 128-byte rows: 16-byte chunk index ^= row % 8;
         // 64-byte rows: chunk index ^= (row / 2) % 4
@@ -701,8 +707,8 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
     constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
     constexpr int kMailMax = TN <= 64 ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox, worst case
-    // Ring depth for a given mailbox size: even, or exactly 3 (every stage then owns an A slot,
-    // which needs a tile of at most 64 tokens).
+    // Ring depth for a given mailbox size: whatever fits (stage s is rebuilt by zip group s % 2, so
+    // odd depths work; they just give the first group one stage more).
     static const int deep_forced = [] {
         const char* e = getenv("DPS_FORCE_DEEP");
         return e ? atoi(e) : -1;
@@ -711,11 +717,15 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     // One CTA per SM with a ring twice as deep when the tiles cannot fill two CTA slots per SM anyway.
     const bool deep = deep_forced >= 0 ? deep_forced != 0 : false;
     const int smem_total = (deep || kCtasPerSm == 1) ? 216 * 1024 : kSmemTotal;
+    static const int max_stages = [] {   // DPS_MAX_STAGES=<n>: tuning knob, caps the ring depth
+        const char* e = getenv("DPS_MAX_STAGES");
+        return e ? atoi(e) : 8;
+    }();
     auto ring_depth = [&](int mail_bytes) {
         int d = (smem_total - mail_bytes) / kStage;
-        if (d > 8) d = 8;
+        if (d > max_stages) d = max_stages;
         if (d < 2) d = 2;
-        if (d % kZipGroups != 0 && !(d == 3 && kZipGroups == 2 && a_slots_max(FULL, TN) >= 3)) d -= d % kZipGroups;
+        if (d >= 6) d &= ~1;   // deep even rings are filled two stages at a time
         return d;
     };
     const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kMailMax + 1024;
@@ -956,8 +966,7 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     int stages = kSmemTotal / kStage;
     if (stages > 8) stages = 8;
     if (stages < 2) stages = 2;
-    if (RB == 1) stages -= stages % kZipGroups;   // stages alternate between the zip groups
-    else if (stages >= 6) stages &= ~1;           // any depth works; even ones fill two stages at a time
+    if (stages >= 6) stages &= ~1;   // any depth works; deep even rings are filled two stages at a time
     const size_t smem = (size_t)stages * kStage + 1024;
     auto kernel = umma_linear_kernel<0, FULL, TN, true, RB>;
     static bool configured = false;
