@@ -85,6 +85,31 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
     return c;
 }
 
+// Activation slots kept apart from the plane ring.  Decode tiles (dense launches, 32 tokens):
+// the activation tile is a third to a fifth of a stage, yet it is needed only when the MMA runs,
+// a DRAM latency after the planes were requested.  Three slots of their own, filled three K blocks
+// ahead of the MMA out of L2, let the same shared memory hold one more plane stage in flight.
+// (Two slots were measured: under load the L2 fetch takes longer than two K blocks, and the MMA
+// warp waited for activations.)  0 = the activation tile travels inside the stage.
+// Not for 64-token tiles: their activation tile is as large as a plane stage, and three slots
+// would leave a ring of two.  Not for 16-token tiles either: measured 2-6 % slower there (the
+// tile is a fifth of a stage, so the slots buy no extra stage).
+#ifndef DPS_XSLOT_MIN_TN
+#define DPS_XSLOT_MIN_TN 32
+#endif
+#ifndef DPS_XSLOT_MAX_TN
+#define DPS_XSLOT_MAX_TN 32
+#endif
+constexpr int kMaxXSlots = 3;
+__host__ __device__ constexpr int x_slots(bool grouped, int tn, int rb) {
+    return (!grouped && rb == 1 && tn >= DPS_XSLOT_MIN_TN && tn <= DPS_XSLOT_MAX_TN) ? kMaxXSlots : 0;
+}
+__host__ __device__ constexpr int x_tile_bytes(bool full, int tn, int rb = 1) { return tn * block_k(full, tn, rb) * 2; }
+// Bytes of one ring stage: planes and activations, or planes alone when the activations have slots.
+__host__ __device__ constexpr int ring_stage_bytes(bool full, int tn, bool grouped, int rb = 1) {
+    return stage_bytes(full, tn, rb) - (x_slots(grouped, tn, rb) ? x_tile_bytes(full, tn, rb) : 0);
+}
+
 // Optional timeline trace (compile with -DDPS_TRACE): lane 0 of each role of CTA (0,0,0) stamps
 // the SM clock at pipeline events of every K block.  Read back with dps_debug_trace().
 #ifdef DPS_TRACE
@@ -133,6 +158,8 @@ struct UmmaParams {
     int num_stages;
     int split;       // K split = cluster size along z; partial tiles are summed through DSMEM
     int red_offset;  // byte offset (from the aligned base of dynamic smem) of the split-K mailbox
+    int x_offset;    // byte offset of the activation slots (tiles whose activations do not ride in the stages)
+    int pair_min;    // ring depth from which stages are filled two at a time
     int* status;
 #ifdef DPS_TRACE
     int trace_slot;  // which half of the CTA time table this launch writes
@@ -245,8 +272,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     constexpr int kXAtoms = kBlockK / 64;    // the x tile is stored as 64-element (128-byte) swizzle atoms
     constexpr int kACols = kBlockK / 2;      // TMEM columns of one A slot (two FP16 per column)
     constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
-    constexpr int kStage = stage_bytes(FULL, TN, RB);
+    constexpr int kStage = ring_stage_bytes(FULL, TN, GROUPED, RB);
     constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
+    constexpr int kXS = x_slots(GROUPED, TN, RB);          // 0 or 3
+    constexpr int kXBytes = x_tile_bytes(FULL, TN, RB);
     constexpr uint32_t kCols = tmem_cols(FULL, TN, RB);
     static_assert(RB == 1 || RB == 2, "one or two row blocks per CTA");
     static_assert(RB == 1 || zip_groups(FULL, TN) == 2, "two row blocks need exactly two zip groups");
@@ -257,6 +286,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     __shared__ __align__(8) uint64_t bar_a_full[kMaxAStages];
     __shared__ __align__(8) uint64_t bar_a_empty[kMaxAStages];
     __shared__ __align__(8) uint64_t bar_d_full;
+    __shared__ __align__(8) uint64_t bar_x_full[kMaxXSlots];
     __shared__ uint32_t tmem_base_slot;
 
     grid_launch_dependents();  // the next kernel's prologue may overlap this kernel's tail
@@ -325,6 +355,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             mbar_init(smem_u32(&bar_a_empty[a]), 1);
         }
         mbar_init(smem_u32(&bar_d_full), 1);
+        for (int a = 0; a < kMaxXSlots; ++a) mbar_init(smem_u32(&bar_x_full[a]), 1);
         fence_barrier_init();
         prefetch_tensormap(&map_p);
         if (FULL) prefetch_tensormap(&map_r);
@@ -352,9 +383,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     bool ok = true;
     if (warp == 0) {
         // ---------------- TMA producer (whole warp converged, one elected lane issues) ----------------
-        // Stages are filled two at a time when the ring is deep enough: the two boxes cover 256
-        // adjacent bytes of every weight row, which DRAM serves noticeably better than 128.
-        const bool pair = (num_stages >= 6) && (num_stages % 2 == 0);
+        // Optionally (tuning knob, off by default) stages are filled two at a time.
+        const bool pair = (num_stages >= prm.pair_min) && (num_stages % 2 == 0);
         // First pass over the ring.  The planes are model state: (dense launches) their loads are
         // issued BEFORE the dependency wait, so that the ring fills while the preceding kernel
         // drains; only the activations -- that kernel's output in a decoder -- wait for it.  A
@@ -368,13 +398,22 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             tma_load_2d(dst, &map_p, full, k, plane_row0);
             if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, plane_row0);
         };
-        auto load_x = [&](int i, int s) {
+        auto load_x = [&](int i, int s) {       // activation tile of K block i, riding in stage s
             const uint32_t full = smem_u32(&bar_full[s]);
             const uint32_t dst = smem_base + (uint32_t)s * kStage;
             const int k = (rank + i * split) * kBlockK;
 #pragma unroll
             for (int t = 0; t < kXAtoms; ++t)
                 tma_load_2d(dst + kXOffset + (uint32_t)(t * TN * 128), &map_x, full, k + t * 64, m0);
+        };
+        auto load_x_slot = [&](int j, int slot) {   // activation tile of K block j into its own slot (j % kXS)
+            const uint32_t full = smem_u32(&bar_x_full[slot]);
+            const uint32_t dst = smem_base + (uint32_t)prm.x_offset + (uint32_t)(slot * kXBytes);
+            const int k = (rank + j * split) * kBlockK;
+            mbar_arrive_expect_tx(full, (uint32_t)kXBytes);
+#pragma unroll
+            for (int t = 0; t < kXAtoms; ++t)
+                tma_load_2d(dst + (uint32_t)(t * TN * 128), &map_x, full, k + t * 64, m0);
         };
         if (!GROUPED && elect_one()) {
             for (int i = 0; i < first; ++i) load_planes(i, i);
@@ -391,18 +430,33 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         DPS_CTA_STAMP_T(8, 0);
         if (!GROUPED) grid_dependency_wait();   // grouped launches waited before reading the tile list
         DPS_CTA_STAMP_T(9, 0);
-        if (elect_one())
-            for (int i = 0; i < first; ++i) {
-                if (GROUPED) load_planes(i, i);
-                load_x(i, i);
+        if (elect_one()) {
+            if (kXS) {
+                for (int j = 0; j < kXS && j < num_kb; ++j) load_x_slot(j, j);
+            } else {
+                for (int i = 0; i < first; ++i) {
+                    if (GROUPED) load_planes(i, i);
+                    load_x(i, i);
+                }
             }
+        }
         __syncwarp();
-        int s = first == num_stages ? 0 : first;
-        uint32_t ph = first == num_stages ? 1u : 0u;
-        for (int i = first; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
-            if (!pair || (i & 1) == 0) {
+        // Steady state.  Without activation slots: wait for stage s to be free, refill it (planes
+        // and activations of K block i).  With slots: the activations of block i - lag, lag =
+        // depth - slots, are requested in the same step as the planes of block i.  Their slot was
+        // last read by the MMA of block i - depth, the very MMA whose completion freed stage s, so
+        // the one wait covers both; the loop runs `lag` steps past the last plane load to request
+        // the remaining activation tiles.
+        const int lag = kXS ? num_stages - kXS : 0;
+        const int begin = kXS ? num_stages : first;
+        int s = begin == num_stages ? 0 : begin;
+        uint32_t ph = begin == num_stages ? 1u : 0u;
+        int xslot = 0;   // slot of block i - lag: the first such block is block kXS, i.e. slot 0 again
+        const int extra = lag > 0 ? lag : 0;   // a ring shallower than the slots makes the lag negative: nothing to add
+        for (int i = begin; i < num_kb + extra && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
+            if (!pair || (i & 1) == 0 || i >= num_kb) {
                 ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);
-                if (ok && pair && i + 1 < num_kb) {     // pairs never wrap: the ring depth is even
+                if (ok && pair && (i & 1) == 0 && i + 1 < num_kb) {     // pairs never wrap: the ring depth is even
                     ok = mbar_wait(smem_u32(&bar_empty[s + 1]), ph ^ 1u);
                 }
             }
@@ -410,8 +464,13 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             if (!ok) break;
             DPS_STAMP(0, i);
             if (elect_one()) {
-                load_planes(i, s);
-                load_x(i, s);
+                if (i < num_kb) load_planes(i, s);
+                if (kXS) {
+                    if (i - lag < num_kb) load_x_slot(i - lag, xslot);
+                    xslot = (xslot + 1 == kXS) ? 0 : xslot + 1;
+                } else {
+                    load_x(i, s);
+                }
             }
             __syncwarp();
         }
@@ -421,8 +480,11 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         int s = 0;
         uint32_t s_parity = 0;
         int cnt[2] = {0, 0};     // K blocks taken from each zip group so far
+        int xslot = 0;           // activation slot of K block i (tiles with activation slots)
+        uint32_t xparity = 0;
         for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
-            const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
+            const uint32_t xbase = kXS ? smem_base + (uint32_t)prm.x_offset + (uint32_t)(xslot * kXBytes)
+                                       : smem_base + (uint32_t)s * kStage + kXOffset;
             if (RB == 2) {
                 // row block g: A slot 2g + (i & 1) of zip group g, accumulator columns [g * TN, (g + 1) * TN)
 #pragma unroll
@@ -464,6 +526,12 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             // activation tile of the stage is complete and visible once a_full is: one wait, not two.
             DPS_STAMP(1, i);
             ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
+            // ... unless the activations have slots of their own: then their barrier is waited for too
+            if (kXS && ok) ok = mbar_wait(smem_u32(&bar_x_full[xslot]), xparity);
+            if (kXS) {
+                xslot = (xslot + 1 == kXS) ? 0 : xslot + 1;
+                xparity ^= (xslot == 0);
+            }
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             DPS_STAMP(2, i);
@@ -650,6 +718,18 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Tuning knob: DPS_PAIR_MIN=<depth> sets the (even) ring depth from which two stages are filled at a
+// time, so that two boxes cover 256 adjacent bytes of every weight row.  Off by default: with rings
+// of 5-7 stages it was measured equal or slower (up to 20 % on a 6-deep full-mode ring) than
+// refilling every stage as soon as it is free.
+int pair_min_depth() {
+    static const int v = [] {
+        const char* e = getenv("DPS_PAIR_MIN");
+        return e ? atoi(e) : 1000;
+    }();
+    return v;
+}
+
 // Tuning / debugging knob: DPS_FORCE_SPLIT=<1..8> pins the K split.
 int forced_split() {
     static const int v = [] {
@@ -701,7 +781,8 @@ int choose_split(int64_t tiles, int total_kb, const int* capacity) {
 template <int ENC, bool FULL, int TN>
 cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y, int64_t M, int64_t N, int64_t K,
                       int* status, cudaStream_t stream) {
-    constexpr int kStage = stage_bytes(FULL, TN);
+    constexpr int kStage = ring_stage_bytes(FULL, TN, false);   // planes only when the activations have slots
+    constexpr int kXRing = x_slots(false, TN, 1) * x_tile_bytes(FULL, TN);
     constexpr int kZipGroups = zip_groups(FULL, TN);
     constexpr int kThreads = cta_threads(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
@@ -722,13 +803,12 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         return e ? atoi(e) : 8;
     }();
     auto ring_depth = [&](int mail_bytes) {
-        int d = (smem_total - mail_bytes) / kStage;
+        int d = (smem_total - mail_bytes - kXRing) / kStage;
         if (d > max_stages) d = max_stages;
         if (d < 2) d = 2;
-        if (d >= 6) d &= ~1;   // deep even rings are filled two stages at a time
         return d;
     };
-    const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kMailMax + 1024;
+    const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kXRing + kMailMax + 1024;
     auto kernel = umma_linear_kernel<ENC, FULL, TN, false>;
     static int capacity[kMaxSplit + 1] = {0};  // per instantiation; filled on first use
     static bool configured = false;
@@ -800,7 +880,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     const int slots = split > 1 ? (TN + split - 1) / split : 0;
     const int mail_bytes = (split > 1 && kMailMax > 0) ? split * slots * kTileRows * 4 : 0;
     const int stages = ring_depth(mail_bytes);
-    const size_t smem = (size_t)stages * kStage + mail_bytes + 1024;
+    const size_t smem = (size_t)stages * kStage + kXRing + mail_bytes + 1024;
     if (kMailMax == 0 && (size_t)stages * kStage < (size_t)TN * kTileRows * 4) split = 1;  // pull mode overlays the ring
     if (getenv("DPS_DEBUG"))
         fprintf(stderr, "[dps] umma TN=%d full=%d N=%lld K=%lld M=%lld stages=%d split=%d capacity=%d,%d,%d,%d,%d,%d,%d,%d\n",
@@ -813,8 +893,10 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     prm.K = (int)K;
     prm.num_stages = stages;
     prm.split = split;
-    prm.red_offset = stages * kStage;
+    prm.x_offset = stages * kStage;
+    prm.red_offset = stages * kStage + kXRing;
     prm.status = status;
+    prm.pair_min = pair_min_depth();
 #ifdef DPS_TRACE
     static int trace_launches = 0;
     prm.trace_slot = (trace_launches++) & 1;
@@ -857,7 +939,6 @@ cudaError_t launch_tn_rb2(const void* x, const uint8_t* p, const uint8_t* r, voi
     int stages = kSmemTotal / kStage;
     if (stages > 8) stages = 8;
     if (stages < 2) stages = 2;
-    if (stages >= 6) stages &= ~1;
     const size_t smem = (size_t)stages * kStage + 1024;
     auto kernel = umma_linear_kernel<ENC, FULL, TN, false, kRb>;
     static bool configured = false;
@@ -892,6 +973,7 @@ cudaError_t launch_tn_rb2(const void* x, const uint8_t* p, const uint8_t* r, voi
     prm.split = 1;
     prm.red_offset = 0;
     prm.status = status;
+    prm.pair_min = pair_min_depth();
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((N + kTileRows * kRb - 1) / (kTileRows * kRb)), (unsigned)((M + TN - 1) / TN), 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
@@ -966,7 +1048,6 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     int stages = kSmemTotal / kStage;
     if (stages > 8) stages = 8;
     if (stages < 2) stages = 2;
-    if (stages >= 6) stages &= ~1;   // any depth works; deep even rings are filled two stages at a time
     const size_t smem = (size_t)stages * kStage + 1024;
     auto kernel = umma_linear_kernel<0, FULL, TN, true, RB>;
     static bool configured = false;
@@ -1003,6 +1084,7 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     prm.split = 1;
     prm.red_offset = 0;
     prm.status = status;
+    prm.pair_min = pair_min_depth();
     GroupedParams gp;
     gp.tiles = static_cast<const int4*>(tiles);
     gp.num_tiles = num_tiles;
