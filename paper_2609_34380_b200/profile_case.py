@@ -4,6 +4,12 @@ Example (one Llama-7B-shaped QKV linear, 8 tokens, fast mode, 4 weight copies so
 planes exceed the L2 capacity):
 
     python -m paper_2609_34380_b200.profile_case --layer qkv --M 8 --mode fast --copies 4 --iters 3
+
+Grouped (MoE) case: --experts E routes --M tokens to two experts each (seeded) over E experts whose
+matrices have --rows output rows (default: the layer's own) and the layer's K:
+
+    python -m paper_2609_34380_b200.profile_case --family mixtral --layer gate_up --experts 8 --rows 7168 \
+        --M 256 --mode fast --iters 3
 """
 from __future__ import annotations
 
@@ -27,7 +33,11 @@ def main() -> None:
     ap.add_argument("--enc", default="auto", choices=["auto", "e4m3", "e5m2"])
     ap.add_argument("--copies", type=int, default=4)
     ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--experts", type=int, default=0, help="> 0: grouped (MoE) linear over this many experts")
+    ap.add_argument("--rows", type=int, default=0, help="grouped case: output rows per expert (0 = the layer's)")
     args = ap.parse_args()
+    if args.experts > 0:
+        return grouped_case(args)
 
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
@@ -63,6 +73,39 @@ def main() -> None:
     nbytes = n * k * (2 if mode else 1) + 2 * args.M * (n + k)
     print(f"{args.family}/{args.layer} N={n} K={k} M={args.M} {args.mode}: {us:.2f} us/launch, "
           f"{nbytes / us / 1e3:.0f} GB/s, {2 * args.M * n * k / us / 1e6:.1f} TFLOP/s, status={dps.dps_stream_status()}")
+
+
+def grouped_case(args) -> None:
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    n, k = SHAPES[args.family][args.layer]
+    n = args.rows or n
+    E, T = args.experts, args.M
+    mode = dps.DPS_MODE_FULL if args.mode == "full" else dps.DPS_MODE_FAST
+    ps, rs, encs = [], [], []
+    for e in range(E):
+        w = workloads.weights(n, k, 4001 + e, device=dev)
+        p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+        ps.append(p), rs.append(r), encs.append(enc)
+        del w
+    P, R = torch.stack(ps), torch.stack(rs)
+    del ps, rs
+    x = workloads.activations(T, k, 4100, device=dev)
+    tor, eor = workloads.top2_routing(T, E, 4200)
+    tor_d, eor_d = torch.from_numpy(tor).to(dev), torch.from_numpy(eor).to(dev)
+    y = torch.empty((2 * T, n), dtype=torch.float16, device=dev)
+    ws = torch.empty(dps.dps_moe_workspace_bytes(2 * T, E, k), dtype=torch.uint8, device=dev)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for it in range(args.iters):
+        if it == args.iters - 1:
+            start.record()
+        dps.dps_moe_linear(mode, encs, x, tor_d, eor_d, P, R if mode else None, y, ws)
+    stop.record()
+    torch.cuda.synchronize()
+    us = 1e3 * start.elapsed_time(stop)
+    nbytes = E * n * k * (2 if mode else 1) + 2 * T * k + 2 * 2 * T * n
+    print(f"{args.family}/{args.layer} grouped E={E} N={n} K={k} tokens={T} {args.mode}: {us:.1f} us/call, "
+          f"{nbytes / us / 1e3:.0f} GB/s, status={dps.dps_stream_status()}")
 
 
 if __name__ == "__main__":
