@@ -179,6 +179,13 @@ struct ZipCtx {
     uint64_t *bar_full, *bar_empty, *bar_a_full, *bar_a_empty;
 };
 
+// Ring position of a zip warp; carried from tile to tile by the persistent kernel.
+struct ZipState {
+    int s = 0;                // stage of the next K block
+    uint32_t s_parity = 0;    // phase parity of that stage
+    int cnt = 0;              // K blocks this warp's group has rebuilt so far
+};
+
 // Zip loop of one warp: for each of its K blocks, wait for the planes to land and for the A slot
 // to be free, rebuild 128 FP16 weights of this thread's row from the plane bytes and store them
 // into tensor memory.  Returns false if a wait timed out.
@@ -186,7 +193,7 @@ struct ZipCtx {
 // RB == 2: the stage holds two row blocks (256 plane rows) that share one activation tile; zip
 // group g rebuilds row block g of EVERY K block into its own two A slots (2g, 2g + 1).
 template <int ENC, bool FULL, int TN, int RB>
-__device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
+__device__ __forceinline__ bool zip_blocks(const ZipCtx& z, ZipState& st) {
     constexpr int kBlockK = block_k(FULL, TN, RB);
     constexpr int kACols = kBlockK / 2;
     constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
@@ -198,10 +205,11 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
     // it uses in turn.
     constexpr int kTotalSlots = a_slots_max(FULL, TN);
     const int my_slots = RB == 2 ? 2 : (kTotalSlots - z.group + 1) / 2;   // 1 or 2
-    int s = 0;
-    uint32_t s_parity = 0;   // phase parity of stage s
-    int cnt = 0;             // K blocks this group has rebuilt so far
-    for (int i = 0; i < z.num_kb && ok; ++i, s = (s + 1 == z.num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
+    int s = st.s;
+    uint32_t s_parity = st.s_parity;   // phase parity of stage s
+    int cnt = st.cnt;                  // K blocks this group has rebuilt so far
+    int i = 0;
+    for (; i < z.num_kb && ok; ++i, s = (s + 1 == z.num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
         if (RB == 1 && (s & 1) != z.group) continue;
         const int turn = my_slots == 2 ? (cnt & 1) : 0;
         const int a = RB == 2 ? 2 * z.group + turn : z.group + 2 * turn;
@@ -256,6 +264,9 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z) {
         }
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(8, i);
     }
+    st.s = s;
+    st.s_parity = s_parity;
+    st.cnt = cnt;
     return ok;
 }
 
@@ -569,9 +580,11 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
         if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2)) {
             // encoding known only at run time (one per expert): uniform branch per CTA
-            ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc);
+            ZipState zst;
+            ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
         } else {
-            ok = zip_blocks<ENC, FULL, TN, RB>(zc);
+            ZipState zst;
+            ok = zip_blocks<ENC, FULL, TN, RB>(zc, zst);
         }
         // E4M3 fast mode multiplied with 2^8 times the weights (hardware FP8 conversion)
         const float out_scale = (!FULL && !e5m2) ? 0.00390625f : 1.0f;
@@ -712,6 +725,292 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     DPS_CTA_STAMP(7);
 }
 
+// ---- persistent variant ----------------------------------------------------------------------
+//
+// One CTA per SM walks a list of tiles.  The three roles run their loops over the same tile
+// sequence without meeting between tiles, so the producer requests the next tile's first stages
+// while the current tile is still being multiplied and drained: set-up, launch gap and the
+// first-load latency are paid once per CTA instead of once per tile.  For the tile shapes that own
+// an SM (256-token full-mode tiles, two-row-block tiles) nothing else would hide them.
+// One accumulator: the MMA warp waits for the epilogue to have read the previous tile out of tensor
+// memory (bar_d_empty) before it starts the next.  The epilogue goes through a small shared-memory
+// buffer (32 token columns at a time), because the stage ring is busy with the next tile.
+// No K split, no activation slots.
+constexpr int kEpiChunkCols = 32;
+
+struct TileCoords {
+    int n0, m0, tile_tokens, plane_row0;
+    bool e5m2;
+};
+
+template <int ENC, int TN, bool GROUPED, int RB>
+__device__ __forceinline__ TileCoords tile_coords(int lin, int row_tiles, int tok_tiles, const UmmaParams& prm,
+                                                  const GroupedParams& gp) {
+    TileCoords t;
+    int row_tile, tok_tile;
+    if (GROUPED) {
+        row_tile = lin % row_tiles;
+        tok_tile = lin / row_tiles;
+    } else if (tok_tiles > 1) {
+        // groups of 8 row tiles x all token tiles (keeps the planes of 8 row tiles and the activation
+        // tiles in L2 while they are in use)
+        constexpr int kRowGroup = 8;
+        const int per_group = kRowGroup * tok_tiles;
+        const int group = lin / per_group, within = lin % per_group;
+        const int rows_here = min(kRowGroup, row_tiles - group * kRowGroup);
+        row_tile = group * kRowGroup + within % rows_here;
+        tok_tile = within / rows_here;
+    } else {
+        row_tile = lin;
+        tok_tile = 0;
+    }
+    t.n0 = row_tile * kTileRows * RB;
+    t.m0 = tok_tile * TN;
+    t.tile_tokens = min(TN, prm.M - t.m0);
+    t.plane_row0 = t.n0;
+    t.e5m2 = (ENC == kEncE5M2);
+    if (GROUPED) {
+        const int4 g = gp.tiles[tok_tile];
+        t.m0 = g.y;
+        t.tile_tokens = g.z;
+        t.plane_row0 = g.x * prm.N + t.n0;
+        t.e5m2 = (gp.e5m2[g.x >> 5] >> (g.x & 31)) & 1u;
+    }
+    return t;
+}
+
+template <int ENC, bool FULL, int TN, bool GROUPED, int RB>
+__global__ void __launch_bounds__(cta_threads(FULL, TN), 1)
+umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
+                       const __grid_constant__ CUtensorMap map_x, const UmmaParams prm, const GroupedParams gp) {
+    constexpr int kBlockK = block_k(FULL, TN, RB);
+    constexpr int kXAtoms = kBlockK / 64;
+    constexpr int kACols = kBlockK / 2;
+    constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
+    constexpr int kStage = stage_bytes(FULL, TN, RB);
+    constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
+    constexpr uint32_t kCols = tmem_cols(FULL, TN, RB);
+    constexpr int kRowsCta = kTileRows * RB;
+    constexpr int kZipGroups = zip_groups(FULL, TN);
+    constexpr int kZipThreads = kZipGroups * 128;
+    constexpr int kTotalSlots = a_slots_max(FULL, TN);
+    static_assert(x_slots(GROUPED, TN, RB) == 0, "the persistent kernel keeps activations in the stages");
+    static_assert(TN % kEpiChunkCols == 0, "tiles are drained 32 token columns at a time");
+
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[kMaxStages];
+    __shared__ __align__(8) uint64_t bar_empty[kMaxStages];
+    __shared__ __align__(8) uint64_t bar_a_full[kMaxAStages];
+    __shared__ __align__(8) uint64_t bar_a_empty[kMaxAStages];
+    __shared__ __align__(8) uint64_t bar_d_full;
+    __shared__ __align__(8) uint64_t bar_d_empty;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    grid_launch_dependents();
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t epi_base = smem_base + (uint32_t)prm.red_offset;   // chunk buffer behind the ring
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_stages = prm.num_stages;
+    const int num_kb = (prm.K + kBlockK - 1) / kBlockK;
+    const int row_tiles = (prm.N + kRowsCta - 1) / kRowsCta;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < num_stages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), RB == 2 ? 9 : 5);
+        }
+        for (int a = 0; a < kMaxAStages; ++a) {
+            mbar_init(smem_u32(&bar_a_full[a]), 4);
+            mbar_init(smem_u32(&bar_a_empty[a]), 1);
+        }
+        mbar_init(smem_u32(&bar_d_full), 1);
+        mbar_init(smem_u32(&bar_d_empty), kZipGroups * 4);   // one arrival per zip warp
+        abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&map_p);
+        if (FULL) prefetch_tensormap(&map_r);
+        prefetch_tensormap(&map_x);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), kCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_slot;
+    const uint32_t tmem_d = tmem_base;
+    const uint32_t tmem_a = tmem_base + RB * TN;
+
+    // Everything read from global memory may come from the preceding kernel (grouped launches: the
+    // tile list does).  These launches run for tens of microseconds at least; fetching planes
+    // ahead of the dependency, as the decode tiles do, would not be noticed.
+    grid_dependency_wait();
+    const int tok_tiles = GROUPED ? *gp.num_tiles : (prm.M + TN - 1) / TN;
+    const int total = row_tiles * tok_tiles;
+    bool ok = true;
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        int s = 0;
+        uint32_t ph = 0;
+        for (int lin = blockIdx.x; lin < total && ok; lin += gridDim.x) {
+            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, row_tiles, tok_tiles, prm, gp);
+            for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
+                ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);   // passes at once on the first ring pass
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                if (elect_one()) {
+                    const uint32_t full = smem_u32(&bar_full[s]);
+                    const uint32_t dst = smem_base + (uint32_t)s * kStage;
+                    const int k = i * kBlockK;
+                    mbar_arrive_expect_tx(full, (uint32_t)kStage);
+                    tma_load_2d(dst, &map_p, full, k, t.plane_row0);
+                    if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, t.plane_row0);
+#pragma unroll
+                    for (int a = 0; a < kXAtoms; ++a)
+                        tma_load_2d(dst + kXOffset + (uint32_t)(a * TN * 128), &map_x, full, k + a * 64, t.m0);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        int s = 0;
+        int cnt[2] = {0, 0};
+        int it = 0;
+        for (int lin = blockIdx.x; lin < total && ok; lin += gridDim.x, ++it) {
+            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, row_tiles, tok_tiles, prm, gp);
+            const int mma_n = GROUPED ? min(TN, (t.tile_tokens + 15) & ~15) : TN;
+            const uint32_t idesc = umma_idesc_f16(kTileRows, mma_n);
+            if (it > 0) {   // the previous tile must have been read out of the accumulator
+                ok = mbar_wait(smem_u32(&bar_d_empty), (uint32_t)(it - 1) & 1u);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+            }
+            for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1) {
+                const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
+#pragma unroll
+                for (int rb = 0; rb < RB; ++rb) {
+                    // RB == 2: zip group rb serves row block rb of every K block; RB == 1: group s % 2
+                    const int g = RB == 2 ? rb : (s & 1);
+                    const int g_slots = RB == 2 ? 2 : (kTotalSlots - g + 1) / 2;
+                    const int turn = g_slots == 2 ? (cnt[g] & 1) : 0;
+                    const int a = RB == 2 ? 2 * g + turn : g + 2 * turn;
+                    const uint32_t a_parity = (uint32_t)(g_slots == 2 ? (cnt[g] >> 1) : cnt[g]) & 1u;
+                    ++cnt[g];
+                    ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int j = 0; j < kBlockK / 16; ++j) {
+                            const uint64_t bdesc = umma_desc_k_sw128(xbase + (uint32_t)((j >> 2) * TN * 128)) +
+                                                   (uint64_t)((j & 3) * 2);
+                            umma_f16_ts(tmem_d + (uint32_t)(rb * TN), tmem_a + (uint32_t)(a * kACols + j * 8), bdesc,
+                                        idesc, (i > 0 || j > 0) ? 1u : 0u);
+                        }
+                        umma_commit(smem_u32(&bar_a_empty[a]));
+                        if (rb == RB - 1) {
+                            umma_commit(smem_u32(&bar_empty[s]));
+                            if (i == num_kb - 1) umma_commit(smem_u32(&bar_d_full));
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+    } else {
+        // ---------------- zip warps: planes -> FP16 -> tensor memory; then the tile's epilogue ----------------
+        const int group = (warp - 2) >> 2;
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        const int zt = (int)threadIdx.x - 64;   // index among the zip threads
+        ZipCtx zc;
+        zc.group = group; zc.warp = warp; zc.lane = lane; zc.row = row;
+        zc.num_kb = num_kb; zc.num_stages = num_stages; zc.stage_bytes = kStage;
+        zc.smem_base = smem_base; zc.tmem_a = tmem_a; zc.lane_base = lane_base;
+        zc.sw = kBlockK == 128 ? (uint32_t)(row & 7) : (uint32_t)((row >> 1) & 3);
+        zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
+        ZipState zst;
+        int it = 0;
+        for (int lin = blockIdx.x; lin < total; lin += gridDim.x, ++it) {
+            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, row_tiles, tok_tiles, prm, gp);
+            if (ok) {
+                if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2))
+                    ok = t.e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
+                else
+                    ok = zip_blocks<ENC, FULL, TN, RB>(zc, zst);
+            }
+            const float out_scale = (!FULL && !t.e5m2) ? 0.00390625f : 1.0f;   // E4M3 fast mode carries 2^8
+            if (ok) ok = mbar_wait(smem_u32(&bar_d_full), (uint32_t)it & 1u);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (ok) tc_fence_after_sync();
+            if (!ok) abort_flag = 1;
+            // The chunk loop has the same trip count for every zip warp (it depends on the tile only),
+            // so the barriers inside always match, also after a timeout somewhere.
+            const int ncols = t.tile_tokens;
+            for (int c0 = 0; c0 < ncols; c0 += kEpiChunkCols) {
+                // drain: RB == 2: this group's row block, all 32 columns; RB == 1: 16 columns per group
+                if (ok) {
+                    const int rb = RB == 2 ? group : 0;
+#pragma unroll
+                    for (int h = 0; h < (RB == 2 ? 2 : 1); ++h) {
+                        const int cb = c0 + (RB == 2 ? 16 * h : 16 * group);
+                        if (cb < ncols) {                     // warp-uniform
+                            uint32_t v[16];
+                            tmem_ld_32x32b_x16(tmem_d + lane_base + (uint32_t)(rb * TN + cb), v);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const __half hv = __float2half_rn(__uint_as_float(v[j]) * out_scale);
+                                const uint32_t addr =
+                                    epi_base + (uint32_t)(((cb - c0 + j) * kRowsCta + rb * kTileRows + row) * 2);
+                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(hv)) : "memory");
+                            }
+                        }
+                    }
+                }
+                if (c0 + kEpiChunkCols >= ncols) {
+                    // last chunk read: the accumulator may be overwritten by the next tile
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_d_empty));
+                }
+                named_barrier_sync(1, kZipThreads);
+                if (ok) {
+                    constexpr int kChunks = kRowsCta / 8;             // 16-byte pieces of one token's rows
+                    const int cols_here = min(kEpiChunkCols, ncols - c0);
+                    for (int item = zt; item < cols_here * kChunks; item += kZipThreads) {
+                        const int c = item / kChunks, qq = item % kChunks;
+                        const int n = t.n0 + qq * 8;
+                        if (n >= prm.N) continue;                     // N is a multiple of 8
+                        const int m = GROUPED ? gp.sorted_rows[t.m0 + c0 + c] : t.m0 + c0 + c;
+                        uint4 val;
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                     : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                                     : "r"(epi_base + (uint32_t)((c * kRowsCta + qq * 8) * 2)));
+                        *reinterpret_cast<uint4*>(prm.y + (int64_t)m * prm.N + n) = val;
+                    }
+                }
+                named_barrier_sync(1, kZipThreads);   // the buffer is free for the next chunk
+            }
+            // after a timeout anywhere among the zip warps they all leave together
+            if (*reinterpret_cast<volatile int*>(&abort_flag)) {
+                ok = false;
+                break;
+            }
+        }
+    }
+    if (!ok) atomicExch(prm.status, (int)DPS_ERR_CUDA);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kCols);
+    }
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -776,6 +1075,61 @@ int choose_split(int64_t tiles, int total_kb, const int* capacity) {
         if (tiles * s <= capacity[s]) best = s;
     }
     return best;
+}
+
+// Tuning knob: DPS_PERSIST=0 launches one CTA per tile even where the persistent kernel applies.
+bool persist_enabled() {
+    static const bool v = [] {
+        const char* e = getenv("DPS_PERSIST");
+        return e ? atoi(e) != 0 : true;
+    }();
+    return v;
+}
+
+// Persistent launch: one CTA per SM (or fewer, if there are fewer tiles) walks `tiles` tiles.
+// prm comes with y, M, N, K, status set; the ring is sized here.
+template <int ENC, bool FULL, int TN, bool GROUPED, int RB>
+cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, const CUtensorMap& mx, UmmaParams prm,
+                              const GroupedParams& gp, int64_t tiles, cudaStream_t stream) {
+    constexpr int kStage = stage_bytes(FULL, TN, RB);
+    constexpr int kEpiBytes = kEpiChunkCols * kTileRows * RB * 2;
+    constexpr int kThreads = cta_threads(FULL, TN);
+    int stages = (216 * 1024 - kEpiBytes) / kStage;
+    if (stages > 8) stages = 8;
+    if (stages < 2) stages = 2;
+    const size_t smem = (size_t)stages * kStage + kEpiBytes + 1024;
+    auto kernel = umma_persistent_kernel<ENC, FULL, TN, GROUPED, RB>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    prm.num_stages = stages;
+    prm.split = 1;
+    prm.red_offset = stages * kStage;   // the epilogue's chunk buffer
+    prm.x_offset = 0;
+    prm.pair_min = pair_min_depth();
+    const int64_t grid = tiles < sm_count() ? tiles : sm_count();
+    if (getenv("DPS_DEBUG"))
+        fprintf(stderr, "[dps] persistent TN=%d full=%d RB=%d grouped=%d tiles<=%lld grid=%lld stages=%d\n", TN, (int)FULL,
+                RB, (int)GROUPED, (long long)tiles, (long long)grid, stages);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, prm, gp);
+    count_launch();
+    return e;
 }
 
 template <int ENC, bool FULL, int TN>
@@ -886,11 +1240,18 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         fprintf(stderr, "[dps] umma TN=%d full=%d N=%lld K=%lld M=%lld stages=%d split=%d capacity=%d,%d,%d,%d,%d,%d,%d,%d\n",
                 TN, (int)FULL, (long long)N, (long long)K, (long long)M, stages, split, capacity[1], capacity[2],
                 capacity[3], capacity[4], capacity[5], capacity[6], capacity[7], capacity[8]);
-    UmmaParams prm;
+    UmmaParams prm = {};
     prm.y = static_cast<__half*>(y);
     prm.M = (int)M;
     prm.N = (int)N;
     prm.K = (int)K;
+    prm.status = status;
+    if constexpr (kCtasPerSm == 1) {
+        // a tile shape that owns its SM: with more tiles than SMs, let one CTA per SM walk them
+        if (split == 1 && persist_enabled() && row_tiles * tok_tiles > sm_count())
+            return launch_persistent<ENC, FULL, TN, false, 1>(mp, mr, mx, prm, GroupedParams{}, row_tiles * tok_tiles,
+                                                             stream);
+    }
     prm.num_stages = stages;
     prm.split = split;
     prm.x_offset = stages * kStage;
@@ -969,10 +1330,15 @@ cudaError_t launch_tn_rb2(const void* x, const uint8_t* p, const uint8_t* r, voi
     prm.M = (int)M;
     prm.N = (int)N;
     prm.K = (int)K;
+    prm.status = status;
+    if constexpr (kCtasPerSm == 1) {
+        const int64_t tiles = ((N + kTileRows * kRb - 1) / (kTileRows * kRb)) * ((M + TN - 1) / TN);
+        if (persist_enabled() && tiles > sm_count())
+            return launch_persistent<ENC, FULL, TN, false, kRb>(mp, mr, mx, prm, GroupedParams{}, tiles, stream);
+    }
     prm.num_stages = stages;
     prm.split = 1;
     prm.red_offset = 0;
-    prm.status = status;
     prm.pair_min = pair_min_depth();
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((N + kTileRows * kRb - 1) / (kTileRows * kRb)), (unsigned)((M + TN - 1) / TN), 1);
@@ -1090,6 +1456,11 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     gp.num_tiles = num_tiles;
     gp.sorted_rows = sorted_rows;
     for (int i = 0; i < 32; ++i) gp.e5m2[i] = e5m2_mask[i];
+    if constexpr (kCtasPerSm == 1 && TN % kEpiChunkCols == 0) {
+        const int64_t upper = ((N + kTileRows * RB - 1) / (kTileRows * RB)) * max_tiles;
+        if (persist_enabled() && upper > sm_count())
+            return launch_persistent<0, FULL, TN, true, RB>(mp, mr, mx, prm, gp, upper, stream);
+    }
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)((N + kTileRows * RB - 1) / (kTileRows * RB)), (unsigned)max_tiles, 1);
