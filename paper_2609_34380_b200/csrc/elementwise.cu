@@ -1,8 +1,8 @@
 // Load-time kernels: tensor statistics for the encoding choice, nested split, reconstruction.
 // Paper: "Mapper: Semi-Unified Memory Abstraction" ("Persistent Region" paragraph) for the
 // split; "Scheduler: Dual-Precision Execution" for the reconstruction and the per-layer
-// encoding choice.  All three are pure streams: 16 elements per thread per step, 128-bit
-// loads and stores, grid sized to the SM count.
+// encoding choice.  All three are pure streams with fully coalesced accesses (consecutive lanes
+// take consecutive 8-weight items, four items per thread in flight), grid sized to the SM count.
 #include "bits.cuh"
 #include "dps_internal.h"
 
@@ -41,34 +41,68 @@ __global__ void __launch_bounds__(kThreads) magnitude_stat_kernel(const uint4* _
     if ((threadIdx.x & 31) == 0 && best) atomicMax(stat, best);
 }
 
+// One item = 8 weights: 16 bytes of FP16 in, 8 bytes of each plane out.  Consecutive lanes take
+// consecutive items, so every warp instruction covers one contiguous span (512 B of loads, 256 B
+// of stores), and four items per thread are in flight per step.
+constexpr int kItemsPerStep = 4;
+
+__device__ __forceinline__ uint2 ldg_stream8(const void* p) {
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
 template <int ENC>
-__global__ void __launch_bounds__(kThreads) split_kernel(const uint4* __restrict__ w, uint4* __restrict__ p,
-                                                         uint4* __restrict__ r, int64_t n16) {
-    for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n16; i += (int64_t)gridDim.x * kThreads) {
-        uint4 a = ldg_stream(w + 2 * i);
-        uint4 b = ldg_stream(w + 2 * i + 1);
-        uint4 pp, rr;
-        split4<ENC>(a.x, a.y, pp.x, rr.x);
-        split4<ENC>(a.z, a.w, pp.y, rr.y);
-        split4<ENC>(b.x, b.y, pp.z, rr.z);
-        split4<ENC>(b.z, b.w, pp.w, rr.w);
-        p[i] = pp;
-        r[i] = rr;
+__global__ void __launch_bounds__(kThreads) split_kernel(const uint4* __restrict__ w, uint2* __restrict__ p,
+                                                         uint2* __restrict__ r, int64_t n8) {
+    const int64_t stride = (int64_t)gridDim.x * kThreads;
+    for (int64_t i0 = blockIdx.x * (int64_t)kThreads + threadIdx.x; i0 < n8; i0 += stride * kItemsPerStep) {
+        uint4 a[kItemsPerStep];
+#pragma unroll
+        for (int u = 0; u < kItemsPerStep; ++u) {
+            const int64_t i = i0 + u * stride;
+            if (i < n8) a[u] = ldg_stream(w + i);
+        }
+#pragma unroll
+        for (int u = 0; u < kItemsPerStep; ++u) {
+            const int64_t i = i0 + u * stride;
+            if (i < n8) {
+                uint2 pp, rr;
+                split4<ENC>(a[u].x, a[u].y, pp.x, rr.x);
+                split4<ENC>(a[u].z, a[u].w, pp.y, rr.y);
+                p[i] = pp;
+                r[i] = rr;
+            }
+        }
     }
 }
 
 template <int ENC, bool FULL>
-__global__ void __launch_bounds__(kThreads) reconstruct_kernel(const uint4* __restrict__ p,
-                                                               const uint4* __restrict__ r, uint4* __restrict__ w,
-                                                               int64_t n16) {
-    for (int64_t i = blockIdx.x * (int64_t)kThreads + threadIdx.x; i < n16; i += (int64_t)gridDim.x * kThreads) {
-        uint4 pp = ldg_stream(p + i);
-        uint4 rr = make_uint4(0, 0, 0, 0);
-        if (FULL) rr = ldg_stream(r + i);
-        uint32_t h[8];
-        join16<ENC, FULL>(pp, rr, h);
-        w[2 * i] = make_uint4(h[0], h[1], h[2], h[3]);
-        w[2 * i + 1] = make_uint4(h[4], h[5], h[6], h[7]);
+__global__ void __launch_bounds__(kThreads) reconstruct_kernel(const uint2* __restrict__ p,
+                                                               const uint2* __restrict__ r, uint4* __restrict__ w,
+                                                               int64_t n8) {
+    const int64_t stride = (int64_t)gridDim.x * kThreads;
+    for (int64_t i0 = blockIdx.x * (int64_t)kThreads + threadIdx.x; i0 < n8; i0 += stride * kItemsPerStep) {
+        uint2 pp[kItemsPerStep], rr[kItemsPerStep];
+#pragma unroll
+        for (int u = 0; u < kItemsPerStep; ++u) {
+            const int64_t i = i0 + u * stride;
+            pp[u] = rr[u] = make_uint2(0, 0);
+            if (i < n8) {
+                pp[u] = ldg_stream8(p + i);
+                if (FULL) rr[u] = ldg_stream8(r + i);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kItemsPerStep; ++u) {
+            const int64_t i = i0 + u * stride;
+            if (i < n8) {
+                uint4 out;
+                join4<ENC, FULL>(pp[u].x, rr[u].x, out.x, out.y);
+                join4<ENC, FULL>(pp[u].y, rr[u].y, out.z, out.w);
+                w[i] = out;
+            }
+        }
     }
 }
 
@@ -94,16 +128,16 @@ cudaError_t launch_magnitude_stat(const uint16_t* w, int64_t n, unsigned* stat, 
 }
 
 cudaError_t launch_split(const uint16_t* w, uint8_t* p, uint8_t* r, int64_t n, int enc, cudaStream_t stream) {
-    int64_t n16 = n / 16;
-    int grid = stream_grid(n16);
+    int64_t n8 = n / 8;
+    int grid = stream_grid((n8 + kItemsPerStep - 1) / kItemsPerStep);
     if (enc == kEncE4M3)
         split_kernel<kEncE4M3><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint4*>(w),
-                                                               reinterpret_cast<uint4*>(p),
-                                                               reinterpret_cast<uint4*>(r), n16);
+                                                               reinterpret_cast<uint2*>(p),
+                                                               reinterpret_cast<uint2*>(r), n8);
     else
         split_kernel<kEncE5M2><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint4*>(w),
-                                                               reinterpret_cast<uint4*>(p),
-                                                               reinterpret_cast<uint4*>(r), n16);
+                                                               reinterpret_cast<uint2*>(p),
+                                                               reinterpret_cast<uint2*>(r), n8);
     count_launch();
     plane_fence_kernel<<<1, 32, 0, stream>>>();
     count_launch();
@@ -112,17 +146,17 @@ cudaError_t launch_split(const uint16_t* w, uint8_t* p, uint8_t* r, int64_t n, i
 
 cudaError_t launch_reconstruct(const uint8_t* p, const uint8_t* r, uint16_t* w, int64_t n, int enc,
                                cudaStream_t stream) {
-    int64_t n16 = n / 16;
-    int grid = stream_grid(n16);
-    const uint4* pp = reinterpret_cast<const uint4*>(p);
-    const uint4* rr = reinterpret_cast<const uint4*>(r);
+    int64_t n8 = n / 8;
+    int grid = stream_grid((n8 + kItemsPerStep - 1) / kItemsPerStep);
+    const uint2* pp = reinterpret_cast<const uint2*>(p);
+    const uint2* rr = reinterpret_cast<const uint2*>(r);
     uint4* ww = reinterpret_cast<uint4*>(w);
     if (enc == kEncE4M3) {
-        if (r) reconstruct_kernel<kEncE4M3, true><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n16);
-        else reconstruct_kernel<kEncE4M3, false><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n16);
+        if (r) reconstruct_kernel<kEncE4M3, true><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
+        else reconstruct_kernel<kEncE4M3, false><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
     } else {
-        if (r) reconstruct_kernel<kEncE5M2, true><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n16);
-        else reconstruct_kernel<kEncE5M2, false><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n16);
+        if (r) reconstruct_kernel<kEncE5M2, true><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
+        else reconstruct_kernel<kEncE5M2, false><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
     }
     count_launch();
     return cudaGetLastError();
