@@ -1,7 +1,8 @@
-"""GPU parity of the two-row-block tiles (256 weight rows per CTA) on small, ragged shapes.
+"""GPU parity of the two-row-block tiles (256 weight rows per CTA) and of the persistent kernel on
+small, ragged shapes.
 
-The launchers pick that tile shape only for large problems; the tuning knobs DPS_DENSE_RB and
-DPS_GROUPED_RB force it.  The library reads its knobs once per process, so the forced run is a child
+The launchers pick those only for large problems; the tuning knobs DPS_DENSE_RB, DPS_GROUPED_RB and
+DPS_PERSIST force them.  The library reads its knobs once per process, so each forced run is a child
 process: this file executed as a script compares against the oracle and prints one line per case.
 """
 import os
@@ -60,13 +61,24 @@ def _cases():
 
 
 @pytest.mark.gpu
-def test_forced_two_row_blocks_in_child_process():
-    env = dict(os.environ, DPS_DENSE_RB="2", DPS_GROUPED_RB="2", PYTHONPATH=REPO)
+@pytest.mark.parametrize("persist", ["0", "2"])      # one CTA per tile / persistent kernel forced
+def test_forced_two_row_blocks_in_child_process(persist):
+    env = dict(os.environ, DPS_DENSE_RB="2", DPS_GROUPED_RB="2", DPS_PERSIST=persist, PYTHONPATH=REPO)
     out = subprocess.run([sys.executable, os.path.abspath(__file__)], cwd=REPO, env=env, capture_output=True,
                          text=True, timeout=600)
     assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-4000:]
     assert "all row-block cases passed" in out.stdout
     assert out.stdout.count("ok dense") == 12 and out.stdout.count("ok grouped") == 4
+
+
+@pytest.mark.gpu
+def test_forced_persistent_kernel_with_default_tiles_in_child_process():
+    """256-token tiles (forced: the shapes here are small) walked by the persistent kernel."""
+    env = dict(os.environ, DPS_PERSIST="2", DPS_FORCE_TN="256", PYTHONPATH=REPO)
+    out = subprocess.run([sys.executable, os.path.abspath(__file__)], cwd=REPO, env=env, capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-4000:]
+    assert "all row-block cases passed" in out.stdout
 
 
 if __name__ == "__main__":
