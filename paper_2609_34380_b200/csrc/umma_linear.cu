@@ -160,6 +160,8 @@ struct UmmaParams {
     int red_offset;  // byte offset (from the aligned base of dynamic smem) of the split-K mailbox
     int x_offset;    // byte offset of the activation slots (tiles whose activations do not ride in the stages)
     int pair_min;    // ring depth from which stages are filled two at a time
+    int tail_parts;  // persistent dense launches: the tiles of the last, partial round are cut into this many
+                     // token ranges (1, 2 or 4), each a work item of its own
     int* status;
 #ifdef DPS_TRACE
     int trace_slot;  // which half of the CTA time table this launch writes
@@ -740,12 +742,29 @@ constexpr int kEpiChunkCols = 32;
 
 struct TileCoords {
     int n0, m0, tile_tokens, plane_row0;
+    int parts;   // 1, 2 or 4: this work item covers TN / parts token columns (activation box of that height)
     bool e5m2;
 };
 
+// Work item `step` of this CTA.  Dense launches: whole tiles blockIdx.x + step * gridDim.x below
+// `t_main` (a multiple of the grid), then ONE more item from the last, partial round, whose tiles
+// are cut into `parts` token ranges so that (almost) every CTA gets a piece instead of a few CTAs a
+// whole tile each.  The pieces write disjoint parts of y: no reduction.  Returns false when done.
+__device__ __forceinline__ bool next_work(int step, int t_main, int total, int parts, int& lin, int& part) {
+    lin = (int)blockIdx.x + step * (int)gridDim.x;
+    part = -1;   // a whole tile
+    if (lin < t_main) return true;
+    if (parts <= 1 || step != t_main / (int)gridDim.x) return false;
+    const int q = (int)blockIdx.x;
+    if (q >= (total - t_main) * parts) return false;
+    lin = t_main + q / parts;
+    part = q % parts;
+    return true;
+}
+
 template <int ENC, int TN, bool GROUPED, int RB>
-__device__ __forceinline__ TileCoords tile_coords(int lin, int row_tiles, int tok_tiles, const UmmaParams& prm,
-                                                  const GroupedParams& gp) {
+__device__ __forceinline__ TileCoords tile_coords(int lin, int part, int parts, int row_tiles, int tok_tiles,
+                                                  const UmmaParams& prm, const GroupedParams& gp) {
     TileCoords t;
     int row_tile, tok_tile;
     if (GROUPED) {
@@ -765,8 +784,9 @@ __device__ __forceinline__ TileCoords tile_coords(int lin, int row_tiles, int to
         tok_tile = 0;
     }
     t.n0 = row_tile * kTileRows * RB;
-    t.m0 = tok_tile * TN;
-    t.tile_tokens = min(TN, prm.M - t.m0);
+    t.parts = part < 0 ? 1 : parts;
+    t.m0 = tok_tile * TN + (part < 0 ? 0 : part * (TN / parts));
+    t.tile_tokens = min(TN / t.parts, prm.M - t.m0);   // may be <= 0 for a piece past the last token: skipped
     t.plane_row0 = t.n0;
     t.e5m2 = (ENC == kEncE5M2);
     if (GROUPED) {
@@ -782,7 +802,9 @@ __device__ __forceinline__ TileCoords tile_coords(int lin, int row_tiles, int to
 template <int ENC, bool FULL, int TN, bool GROUPED, int RB>
 __global__ void __launch_bounds__(cta_threads(FULL, TN), 1)
 umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
-                       const __grid_constant__ CUtensorMap map_x, const UmmaParams prm, const GroupedParams gp) {
+                       const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_x2,
+                       const __grid_constant__ CUtensorMap map_x4, const UmmaParams prm, const GroupedParams gp) {
+    // map_x2 / map_x4: the activation matrix again, with boxes of TN / 2 and TN / 4 rows (tail pieces)
     constexpr int kBlockK = block_k(FULL, TN, RB);
     constexpr int kXAtoms = kBlockK / 64;
     constexpr int kACols = kBlockK / 2;
@@ -846,13 +868,19 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     grid_dependency_wait();
     const int tok_tiles = GROUPED ? *gp.num_tiles : (prm.M + TN - 1) / TN;
     const int total = row_tiles * tok_tiles;
+    const int parts = GROUPED ? 1 : prm.tail_parts;
+    const int t_main = parts > 1 ? (total / (int)gridDim.x) * (int)gridDim.x : total;
     bool ok = true;
+    int lin, part;
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         int s = 0;
         uint32_t ph = 0;
-        for (int lin = blockIdx.x; lin < total && ok; lin += gridDim.x) {
-            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, row_tiles, tok_tiles, prm, gp);
+        for (int step = 0; ok && next_work(step, t_main, total, parts, lin, part); ++step) {
+            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
+            if (t.tile_tokens <= 0) continue;
+            const CUtensorMap* xmap = t.parts == 4 ? &map_x4 : t.parts == 2 ? &map_x2 : &map_x;
+            const uint32_t stage_tx = (uint32_t)(kStage - (TN - TN / t.parts) * kBlockK * 2);
             for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
                 ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);   // passes at once on the first ring pass
                 ok = __all_sync(0xFFFFFFFFu, ok);
@@ -861,12 +889,12 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                     const uint32_t full = smem_u32(&bar_full[s]);
                     const uint32_t dst = smem_base + (uint32_t)s * kStage;
                     const int k = i * kBlockK;
-                    mbar_arrive_expect_tx(full, (uint32_t)kStage);
+                    mbar_arrive_expect_tx(full, stage_tx);
                     tma_load_2d(dst, &map_p, full, k, t.plane_row0);
                     if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, t.plane_row0);
 #pragma unroll
                     for (int a = 0; a < kXAtoms; ++a)
-                        tma_load_2d(dst + kXOffset + (uint32_t)(a * TN * 128), &map_x, full, k + a * 64, t.m0);
+                        tma_load_2d(dst + kXOffset + (uint32_t)(a * TN * 128), xmap, full, k + a * 64, t.m0);
                 }
                 __syncwarp();
             }
@@ -876,9 +904,11 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         int s = 0;
         int cnt[2] = {0, 0};
         int it = 0;
-        for (int lin = blockIdx.x; lin < total && ok; lin += gridDim.x, ++it) {
-            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, row_tiles, tok_tiles, prm, gp);
-            const int mma_n = GROUPED ? min(TN, (t.tile_tokens + 15) & ~15) : TN;
+        for (int step = 0; ok && next_work(step, t_main, total, parts, lin, part); ++step) {
+            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
+            if (t.tile_tokens <= 0) continue;
+            // UMMA N: only the token columns the item has, rounded up to 16
+            const int mma_n = min(TN, (t.tile_tokens + 15) & ~15);
             const uint32_t idesc = umma_idesc_f16(kTileRows, mma_n);
             if (it > 0) {   // the previous tile must have been read out of the accumulator
                 ok = mbar_wait(smem_u32(&bar_d_empty), (uint32_t)(it - 1) & 1u);
@@ -918,6 +948,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                     __syncwarp();
                 }
             }
+            ++it;
         }
     } else {
         // ---------------- zip warps: planes -> FP16 -> tensor memory; then the tile's epilogue ----------------
@@ -934,8 +965,9 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
         ZipState zst;
         int it = 0;
-        for (int lin = blockIdx.x; lin < total; lin += gridDim.x, ++it) {
-            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, row_tiles, tok_tiles, prm, gp);
+        for (int step = 0; next_work(step, t_main, total, parts, lin, part); ++step) {
+            const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
+            if (t.tile_tokens <= 0) continue;
             if (ok) {
                 if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2))
                     ok = t.e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
@@ -995,6 +1027,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                 }
                 named_barrier_sync(1, kZipThreads);   // the buffer is free for the next chunk
             }
+            ++it;
             // after a timeout anywhere among the zip warps they all leave together
             if (*reinterpret_cast<volatile int*>(&abort_flag)) {
                 ok = false;
@@ -1091,9 +1124,12 @@ bool use_persistent(int64_t tiles) { return persist_mode() == 2 || (persist_mode
 
 // Persistent launch: one CTA per SM (or fewer, if there are fewer tiles) walks `tiles` tiles.
 // prm comes with y, M, N, K, status set; the ring is sized here.
+// x / x_rows: the activation matrix (dense launches), needed for the half- and quarter-height
+// boxes of the tail pieces.
 template <int ENC, bool FULL, int TN, bool GROUPED, int RB>
 cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, const CUtensorMap& mx, UmmaParams prm,
-                              const GroupedParams& gp, int64_t tiles, cudaStream_t stream) {
+                              const GroupedParams& gp, int64_t tiles, const void* x, int64_t x_rows,
+                              cudaStream_t stream) {
     constexpr int kStage = stage_bytes(FULL, TN, RB);
     constexpr int kEpiBytes = kEpiChunkCols * kTileRows * RB * 2;
     constexpr int kThreads = cta_threads(FULL, TN);
@@ -1117,9 +1153,37 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
     prm.x_offset = 0;
     prm.pair_min = pair_min_depth();
     const int64_t grid = tiles < sm_count() ? tiles : sm_count();
+    // Last, partial round of a dense launch: cut its tiles into 2 or 4 token ranges if that gives
+    // more CTAs something to do (each piece streams the tile's planes again, out of L2, but
+    // multiplies and fetches only its share of the activations).  Measured gain: 0-4 % -- the
+    // weight-side work (plane loads, rebuilding) of a piece is that of a whole tile.
+    // DPS_TAIL_PARTS=1|2|4 overrides.
+    static const int parts_forced = [] {
+        const char* e = getenv("DPS_TAIL_PARTS");
+        return e ? atoi(e) : 0;
+    }();
+    int parts = 1;
+    CUtensorMap mx2 = mx, mx4 = mx;
+    if (!GROUPED) {
+        const int64_t tail = tiles % grid;
+        if (tail > 0 && tiles > grid) {
+            if (2 * tail <= grid) parts = 2;
+            if (4 * tail <= grid) parts = 4;
+        }
+        if ((parts_forced == 1 || parts_forced == 2 || parts_forced == 4) && tail * parts_forced <= grid)
+            parts = tiles > grid ? parts_forced : 1;   // every piece of the tail needs a CTA of its own
+        if (parts > 1) {
+            if (!make_map_2d(&mx2, x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)x_rows, (uint64_t)prm.K, TN / 2, 64,
+                             CU_TENSOR_MAP_SWIZZLE_128B) ||
+                !make_map_2d(&mx4, x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)x_rows, (uint64_t)prm.K, TN / 4, 64,
+                             CU_TENSOR_MAP_SWIZZLE_128B))
+                return cudaErrorInvalidValue;
+        }
+    }
+    prm.tail_parts = parts;
     if (getenv("DPS_DEBUG"))
-        fprintf(stderr, "[dps] persistent TN=%d full=%d RB=%d grouped=%d tiles<=%lld grid=%lld stages=%d\n", TN, (int)FULL,
-                RB, (int)GROUPED, (long long)tiles, (long long)grid, stages);
+        fprintf(stderr, "[dps] persistent TN=%d full=%d RB=%d grouped=%d tiles<=%lld grid=%lld stages=%d tail_parts=%d\n",
+                TN, (int)FULL, RB, (int)GROUPED, (long long)tiles, (long long)grid, stages, parts);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
@@ -1130,7 +1194,7 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, prm, gp);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, mx2, mx4, prm, gp);
     count_launch();
     return e;
 }
@@ -1253,7 +1317,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         // a tile shape that owns its SM: with more tiles than SMs, let one CTA per SM walk them
         if (split == 1 && use_persistent(row_tiles * tok_tiles))
             return launch_persistent<ENC, FULL, TN, false, 1>(mp, mr, mx, prm, GroupedParams{}, row_tiles * tok_tiles,
-                                                             stream);
+                                                             x, M, stream);
     }
     prm.num_stages = stages;
     prm.split = split;
@@ -1337,7 +1401,7 @@ cudaError_t launch_tn_rb2(const void* x, const uint8_t* p, const uint8_t* r, voi
     if constexpr (kCtasPerSm == 1) {
         const int64_t tiles = ((N + kTileRows * kRb - 1) / (kTileRows * kRb)) * ((M + TN - 1) / TN);
         if (use_persistent(tiles))
-            return launch_persistent<ENC, FULL, TN, false, kRb>(mp, mr, mx, prm, GroupedParams{}, tiles, stream);
+            return launch_persistent<ENC, FULL, TN, false, kRb>(mp, mr, mx, prm, GroupedParams{}, tiles, x, M, stream);
     }
     prm.num_stages = stages;
     prm.split = 1;
@@ -1466,7 +1530,7 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     if constexpr (kCtasPerSm == 1 && TN % kEpiChunkCols == 0) {
         const int64_t upper = ((N + kTileRows * RB - 1) / (kTileRows * RB)) * max_tiles;
         if (use_persistent(upper))
-            return launch_persistent<0, FULL, TN, true, RB>(mp, mr, mx, prm, gp, upper, stream);
+            return launch_persistent<0, FULL, TN, true, RB>(mp, mr, mx, prm, gp, upper, x_sorted, A, stream);
     }
 
     cudaLaunchConfig_t cfg = {};
