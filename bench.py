@@ -413,6 +413,16 @@ def detail_rows(dps, workloads, torch, dev, peaks):
     stream = torch.cuda.Stream(device=dev)
     hbm, tc = peaks["hbm_gbs"], peaks["bf16_tflops"]
 
+    # ---- this GPU's own copy bandwidth, same run (context for the fractions: the denominator in
+    #      `peaks` was measured on one B200 of the pool, and the GPUs differ by a few per cent) ----
+    src = torch.zeros(1 << 28, dtype=torch.float32, device=dev)
+    dst = torch.empty_like(src)
+    ms, _ = _time_graph(torch, stream, lambda: [torch.add(src, 1.0, out=dst) for _ in range(4)])
+    nbytes = 4 * 2 * src.numel() * 4
+    out["device_copy_probe"] = {"GB/s": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes,
+                                "what": "4 x (1 GiB read + 1 GiB written) by an elementwise torch kernel, CUDA-graph replay"}
+    del src, dst
+
     # ---- split / reconstruct: 8 gate+up-shaped tensors (1.4 GB of FP16, larger than L2) ----
     n, k = workloads.LLAMA7B["gate_up"]
     ws = [workloads.weights(n, k, 2003 + 100 * c, device=dev) for c in range(8)]
