@@ -17,6 +17,7 @@
 
 #include "dps_internal.h"
 #include "gemv.cuh"
+#include "sm100.cuh"
 
 namespace dps {
 
@@ -70,6 +71,9 @@ moe_route_kernel(const int32_t* __restrict__ token_of_row, const int32_t* __rest
                  int32_t* num_tiles, int4* tiles, int* status) {
     __shared__ int s_cnt[kMaxExperts];
     __shared__ int s_off[kMaxExperts];
+    // the gather and the grouped kernel may be made resident now; both wait for their predecessor
+    // (griddepcontrol.wait) before they read anything this kernel writes
+    sm100::grid_launch_dependents();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int bad = 0;
     for (int a = tid; a < A; a += kRouteThreads) bad |= !row_valid(token_of_row, expert_of_row, a, T, E);
@@ -118,6 +122,8 @@ __global__ void __launch_bounds__(256)
 moe_gather_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ token_of_row,
                   const int32_t* __restrict__ sorted_rows, const int32_t* __restrict__ num_tiles,
                   uint4* __restrict__ x_sorted, int64_t k16) {
+    sm100::grid_launch_dependents();
+    sm100::grid_dependency_wait();   // sorted_rows and num_tiles come from the routing kernel
     const int valid = num_tiles[1];
     for (int i = blockIdx.x; i < valid; i += gridDim.x) {
         const int a = sorted_rows[i];
@@ -147,11 +153,22 @@ cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const i
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     const int gather_grid = (int)(A < 4096 ? A : 4096);
-    moe_gather_kernel<<<gather_grid, 256, 0, stream>>>(static_cast<const uint4*>(x), token_of_row, w.sorted_rows,
-                                                      w.num_tiles, reinterpret_cast<uint4*>(w.x_sorted), K / 8);
-    count_launch();
-    err = cudaGetLastError();
-    if (err != cudaSuccess) return err;
+    {   // programmatic dependent launch: resident while the routing kernel runs, waits before its first read
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)gather_grid, 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        err = cudaLaunchKernelEx(&cfg, moe_gather_kernel, static_cast<const uint4*>(x), token_of_row,
+                                 (const int32_t*)w.sorted_rows, (const int32_t*)w.num_tiles,
+                                 reinterpret_cast<uint4*>(w.x_sorted), (int64_t)(K / 8));
+        count_launch();
+        if (err != cudaSuccess) return err;
+    }
 
     uint32_t mask[kMaxExperts / 32];
     for (int i = 0; i < kMaxExperts / 32; ++i) mask[i] = 0;
