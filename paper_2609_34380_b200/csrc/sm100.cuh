@@ -197,6 +197,15 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
     return v;
 }
 
+__device__ __forceinline__ float4 ld_cluster_v4_f32(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(addr)
+                 : "memory");
+    return v;
+}
+
 // ---- programmatic dependent launch ---------------------------------------------------------------
 // launch_dependents: the next kernel in the stream (if launched with programmatic stream
 // serialization) may begin once every CTA of this grid has executed this or exited.

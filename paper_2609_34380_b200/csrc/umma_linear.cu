@@ -746,15 +746,30 @@ struct TileCoords {
     bool e5m2;
 };
 
-// Work item `step` of this CTA.  Dense launches: whole tiles blockIdx.x + step * gridDim.x below
-// `t_main` (a multiple of the grid), then ONE more item from the last, partial round, whose tiles
-// are cut into `parts` token ranges so that (almost) every CTA gets a piece instead of a few CTAs a
-// whole tile each.  The pieces write disjoint parts of y: no reduction.  Returns false when done.
-__device__ __forceinline__ bool next_work(int step, int t_main, int total, int parts, int& lin, int& part) {
+// Work item `step` of this CTA: whole tiles blockIdx.x + step * gridDim.x below `t_main`, then ONE
+// more item from the last, partial round, in which otherwise a few CTAs would get a whole tile each
+// and the rest nothing:
+//   * `ksplit` (CTA pairs launched as clusters of two, at most half as many tiles left as CTAs): pair p
+//     takes tile t_main + p and each CTA of it one half of K (khalf = its rank); the halves are summed
+//     through the pair's shared memory at the very end;
+//   * else `parts` > 1 (dense launches): the tiles are cut into `parts` token ranges (part), which
+//     write disjoint parts of y.
+// Returns false when the CTA is done.
+__device__ __forceinline__ bool next_work(int step, int t_main, int total, int parts, bool ksplit, int& lin, int& part,
+                                          int& khalf) {
     lin = (int)blockIdx.x + step * (int)gridDim.x;
-    part = -1;   // a whole tile
+    part = -1;    // a whole tile
+    khalf = -1;   // all of K
     if (lin < t_main) return true;
-    if (parts <= 1 || step != t_main / (int)gridDim.x) return false;
+    if (step != t_main / (int)gridDim.x) return false;
+    if (ksplit) {
+        const int pair = (int)blockIdx.x >> 1;
+        if (pair >= total - t_main) return false;
+        lin = t_main + pair;
+        khalf = (int)blockIdx.x & 1;
+        return true;
+    }
+    if (parts <= 1) return false;
     const int q = (int)blockIdx.x;
     if (q >= (total - t_main) * parts) return false;
     lin = t_main + q / parts;
@@ -868,27 +883,35 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     grid_dependency_wait();
     const int tok_tiles = GROUPED ? *gp.num_tiles : (prm.M + TN - 1) / TN;
     const int total = row_tiles * tok_tiles;
-    const int parts = GROUPED ? 1 : prm.tail_parts;
-    const int t_main = parts > 1 ? (total / (int)gridDim.x) * (int)gridDim.x : total;
+    // Last, partial round: halves of K for CTA pairs if the launch came as clusters of two and there
+    // are at most half as many tiles left as CTAs; else token ranges (dense launches, if asked for).
+    const int tail_tiles = total % (int)gridDim.x;
+    const bool ksplit = prm.split == 2 && tail_tiles > 0 && 2 * tail_tiles <= (int)gridDim.x && num_kb >= 2;
+    const int parts = (GROUPED || ksplit) ? 1 : prm.tail_parts;
+    const int t_main = (ksplit || parts > 1) ? total - tail_tiles : total;
+    const bool has_khalf = ksplit && ((int)blockIdx.x >> 1) < tail_tiles;   // same for both CTAs of a pair
     bool ok = true;
-    int lin, part;
+    int lin, part, khalf;
+    int last_ncols = 0, last_n0 = 0, last_m0 = 0;   // the K-half item's tile, for the pair's reduction below
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         int s = 0;
         uint32_t ph = 0;
-        for (int step = 0; ok && next_work(step, t_main, total, parts, lin, part); ++step) {
+        for (int step = 0; ok && next_work(step, t_main, total, parts, ksplit, lin, part, khalf); ++step) {
             const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
             if (t.tile_tokens <= 0) continue;
             const CUtensorMap* xmap = t.parts == 4 ? &map_x4 : t.parts == 2 ? &map_x2 : &map_x;
             const uint32_t stage_tx = (uint32_t)(kStage - (TN - TN / t.parts) * kBlockK * 2);
-            for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
+            const int kb0 = khalf == 1 ? num_kb / 2 : 0;
+            const int nkb = khalf < 0 ? num_kb : (khalf == 0 ? num_kb / 2 : num_kb - num_kb / 2);
+            for (int i = 0; i < nkb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
                 ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);   // passes at once on the first ring pass
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 if (elect_one()) {
                     const uint32_t full = smem_u32(&bar_full[s]);
                     const uint32_t dst = smem_base + (uint32_t)s * kStage;
-                    const int k = i * kBlockK;
+                    const int k = (kb0 + i) * kBlockK;
                     mbar_arrive_expect_tx(full, stage_tx);
                     tma_load_2d(dst, &map_p, full, k, t.plane_row0);
                     if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, t.plane_row0);
@@ -904,9 +927,10 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         int s = 0;
         int cnt[2] = {0, 0};
         int it = 0;
-        for (int step = 0; ok && next_work(step, t_main, total, parts, lin, part); ++step) {
+        for (int step = 0; ok && next_work(step, t_main, total, parts, ksplit, lin, part, khalf); ++step) {
             const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
             if (t.tile_tokens <= 0) continue;
+            const int nkb = khalf < 0 ? num_kb : (khalf == 0 ? num_kb / 2 : num_kb - num_kb / 2);
             // UMMA N: only the token columns the item has, rounded up to 16
             const int mma_n = min(TN, (t.tile_tokens + 15) & ~15);
             const uint32_t idesc = umma_idesc_f16(kTileRows, mma_n);
@@ -916,7 +940,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                 if (!ok) break;
                 tc_fence_after_sync();
             }
-            for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1) {
+            for (int i = 0; i < nkb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1) {
                 const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
 #pragma unroll
                 for (int rb = 0; rb < RB; ++rb) {
@@ -942,7 +966,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                         umma_commit(smem_u32(&bar_a_empty[a]));
                         if (rb == RB - 1) {
                             umma_commit(smem_u32(&bar_empty[s]));
-                            if (i == num_kb - 1) umma_commit(smem_u32(&bar_d_full));
+                            if (i == nkb - 1) umma_commit(smem_u32(&bar_d_full));
                         }
                     }
                     __syncwarp();
@@ -965,9 +989,10 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
         ZipState zst;
         int it = 0;
-        for (int step = 0; next_work(step, t_main, total, parts, lin, part); ++step) {
+        for (int step = 0; next_work(step, t_main, total, parts, ksplit, lin, part, khalf); ++step) {
             const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
             if (t.tile_tokens <= 0) continue;
+            zc.num_kb = khalf < 0 ? num_kb : (khalf == 0 ? num_kb / 2 : num_kb - num_kb / 2);
             if (ok) {
                 if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2))
                     ok = t.e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
@@ -979,9 +1004,30 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (ok) tc_fence_after_sync();
             if (!ok) abort_flag = 1;
+            const int ncols = t.tile_tokens;
+            if (khalf >= 0) {
+                // Half of K (always this CTA's last item): the FP32 partial tile goes to shared memory,
+                // red[token][row], over the ring -- nothing is in flight any more -- and the pair sums
+                // the halves after the role loops.
+                last_ncols = ncols; last_n0 = t.n0; last_m0 = t.m0;
+                if (ok) {
+                    const int rb = RB == 2 ? group : 0;
+                    for (int cb = (RB == 2 ? 0 : 16 * group); cb < ncols; cb += (RB == 2 ? 16 : 32)) {
+                        uint32_t v[16];
+                        tmem_ld_32x32b_x16(tmem_d + lane_base + (uint32_t)(rb * TN + cb), v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const uint32_t addr = smem_base + (uint32_t)(((cb + j) * kRowsCta + rb * kTileRows + row) * 4);
+                            asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(__uint_as_float(v[j]) * out_scale)
+                                         : "memory");
+                        }
+                    }
+                }
+                break;
+            }
             // The chunk loop has the same trip count for every zip warp (it depends on the tile only),
             // so the barriers inside always match, also after a timeout somewhere.
-            const int ncols = t.tile_tokens;
             for (int c0 = 0; c0 < ncols; c0 += kEpiChunkCols) {
                 // drain: RB == 2: this group's row block, all 32 columns; RB == 1: 16 columns per group
                 if (ok) {
@@ -1036,6 +1082,41 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         }
     }
     if (!ok) atomicExch(prm.status, (int)DPS_ERR_CUDA);
+    if (has_khalf) {
+        // ---- the pair sums its two halves of K: every CTA takes the 8-row pieces of its parity, adds
+        //      the peer's partial (read out of the peer's shared memory) to its own, writes FP16 ----
+        __shared__ int s_tile[3];
+        if (threadIdx.x == 64) { s_tile[0] = last_ncols; s_tile[1] = last_n0; s_tile[2] = last_m0; }   // a zip thread knows
+        __syncthreads();
+        cluster_sync_all();   // both partial tiles are complete and visible
+        const int ncols = s_tile[0], n0 = s_tile[1], m0 = s_tile[2];
+        const uint32_t rank = cluster_ctarank();
+        // CTA `rank` takes the tokens of its parity; consecutive threads take consecutive 8-row pieces
+        // of a token (32 contiguous bytes each, two 16-byte loads from each partial tile)
+        constexpr int kPieces = kRowsCta / 8;
+        const int my_cols = (ncols - (int)rank + 1) / 2;
+        for (int idx = (int)threadIdx.x; idx < my_cols * kPieces; idx += cta_threads(FULL, TN)) {
+            const int c = (int)rank + 2 * (idx / kPieces), qq = idx % kPieces;
+            const int n = n0 + qq * 8;
+            if (n >= prm.N) continue;
+            const uint32_t local = smem_base + (uint32_t)((c * kRowsCta + qq * 8) * 4);
+            const uint32_t remote = map_to_cta(local, rank ^ 1u);
+            float4 a0, a1;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                         : "=f"(a0.x), "=f"(a0.y), "=f"(a0.z), "=f"(a0.w) : "r"(local));
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                         : "=f"(a1.x), "=f"(a1.y), "=f"(a1.z), "=f"(a1.w) : "r"(local + 16u));
+            const float4 b0 = ld_cluster_v4_f32(remote), b1 = ld_cluster_v4_f32(remote + 16u);
+            const int m = GROUPED ? gp.sorted_rows[m0 + c] : m0 + c;
+            uint4 out;
+            out.x = pack_half2(a0.x + b0.x, a0.y + b0.y);
+            out.y = pack_half2(a0.z + b0.z, a0.w + b0.w);
+            out.z = pack_half2(a1.x + b1.x, a1.y + b1.y);
+            out.w = pack_half2(a1.z + b1.z, a1.w + b1.w);
+            *reinterpret_cast<uint4*>(prm.y + (int64_t)m * prm.N + n) = out;
+        }
+        cluster_sync_all();   // nobody leaves while its peer may still read its partial tile
+    }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
@@ -1148,11 +1229,21 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
         configured = true;
     }
     prm.num_stages = stages;
-    prm.split = 1;
     prm.red_offset = stages * kStage;   // the epilogue's chunk buffer
     prm.x_offset = 0;
     prm.pair_min = pair_min_depth();
-    const int64_t grid = tiles < sm_count() ? tiles : sm_count();
+    int64_t grid = tiles < sm_count() ? tiles : sm_count();
+    // CTA pairs (clusters of two) so that the tiles of a short last round can be shared out as halves
+    // of K, summed through the pair's shared memory; the FP32 partial tile must fit over the ring.
+    // DPS_TAIL_KSPLIT=0 launches single CTAs (tuning knob).
+    static const int ksplit_mode = [] {   // 2: pairs launched, no split (isolates the cost of the cluster launch)
+        const char* e = getenv("DPS_TAIL_KSPLIT");
+        return e ? atoi(e) : 1;
+    }();
+    const bool ksplit_enabled = ksplit_mode != 0;
+    const bool pairs = ksplit_enabled && grid >= 2 && (size_t)TN * kTileRows * RB * 4 <= (size_t)stages * kStage;
+    if (pairs) grid &= ~(int64_t)1;
+    prm.split = (pairs && ksplit_mode == 1) ? 2 : 1;
     // Last, partial round of a dense launch: cut its tiles into 2 or 4 token ranges if that gives
     // more CTAs something to do (each piece streams the tile's planes again, out of L2, but
     // multiplies and fetches only its share of the activations).  Measured gain: 0-4 % -- the
@@ -1166,7 +1257,7 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
     CUtensorMap mx2 = mx, mx4 = mx;
     if (!GROUPED) {
         const int64_t tail = tiles % grid;
-        if (tail > 0 && tiles > grid) {
+        if (!pairs && tail > 0 && tiles > grid) {   // with CTA pairs the short last round is split along K instead
             if (2 * tail <= grid) parts = 2;
             if (4 * tail <= grid) parts = 4;
         }
@@ -1182,18 +1273,22 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
     }
     prm.tail_parts = parts;
     if (getenv("DPS_DEBUG"))
-        fprintf(stderr, "[dps] persistent TN=%d full=%d RB=%d grouped=%d tiles<=%lld grid=%lld stages=%d tail_parts=%d\n",
-                TN, (int)FULL, RB, (int)GROUPED, (long long)tiles, (long long)grid, stages, parts);
+        fprintf(stderr, "[dps] persistent TN=%d full=%d RB=%d grouped=%d tiles<=%lld grid=%lld stages=%d tail_parts=%d pairs=%d\n",
+                TN, (int)FULL, RB, (int)GROUPED, (long long)tiles, (long long)grid, stages, parts, (int)pairs);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pairs ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mr, mx, mx2, mx4, prm, gp);
     count_launch();
     return e;
