@@ -1536,13 +1536,13 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
         const char* e = getenv("DPS_DENSE_RB");
         return e ? atoi(e) : 0;
     }();
-    // Fast mode with enough tiles to give every SM one and a half: 256 weight rows per CTA share
+    // Fast mode with more such tiles than SMs (the persistent kernel then walks them): 256 weight rows per CTA share
     // each 128-token activation tile, which halves the activation bytes pulled out of L2 per
     // FLOP (measured +2-8 % at 2048-8192 tokens; with fewer tiles the SMs run dry, and in full
     // mode the zip warps would rebuild twice the weights per MMA cycle: -20 %).
     // DPS_DENSE_RB=1|2 overrides (tuning knob).
     const int64_t tiles_rb2 = ((N + 2 * kTileRows - 1) / (2 * kTileRows)) * ((M + 127) / 128);
-    const bool rb2 = rb_forced ? rb_forced == 2 : (!FULL && 2 * tiles_rb2 >= 3 * (int64_t)sm_count());
+    const bool rb2 = rb_forced ? rb_forced == 2 : (!FULL && tiles_rb2 > (int64_t)sm_count());
     if (rb2 && M > 64) return launch_tn_rb2<ENC, FULL, 128>(x, p, r, y, M, N, K, status, stream);
     // ... unless 256-token tiles would leave half the SMs without one (few weight rows, few tokens):
     // then 128-token tiles, two CTAs per SM, win by 10-40 % (measured at 256 tokens, N = 4096 / 8192).
