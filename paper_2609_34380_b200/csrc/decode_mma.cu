@@ -74,16 +74,18 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
     constexpr float kScale = (ENC == kEncE4M3 && !FULL) ? 0.00390625f : 1.0f;  // 2^-8, exact
     __shared__ float red[kWarps][kRowsPerBlock][NT * 8 + 1];
     sm100::grid_launch_dependents();
-    // A CTA that becomes resident while the preceding kernel drains has nothing to compute with yet
-    // (its activations are that kernel's output), but its weights are model state: ask L2 for the
-    // CTA's row block now, so that the DRAM pipe keeps working through the other kernel's tail and
-    // the loads below hit L2.  Thread i takes row i / 16 and every 16th 128-byte line of it.
+    // A CTA that becomes resident while the preceding kernel drains has no activations yet (they are
+    // that kernel's output), but its weights are model state: the first batch of weight loads is
+    // issued BEFORE the dependency wait (below), and the first wave of CTAs asks L2 for the stretch
+    // of its rows behind that batch, so that the DRAM pipe keeps working through the other
+    // kernel's tail.  Thread i takes row i / 16 and every 16th 128-byte line of it.
     if (prefetch_steps > 0 && (int)blockIdx.x < prefetch_ctas) {
         const int64_t prow = (int64_t)blockIdx.x * (HALF ? 8 : kRowsPerBlock) + (threadIdx.x >> 4);
         if (prow < N && (!HALF || (threadIdx.x >> 4) < 8)) {
-            const int64_t pbase = prow * K + (threadIdx.x & 15) * 128;
+            const int64_t first = (int64_t)U * kRoundK;   // bytes of a row the first batch loads itself
+            const int64_t pbase = prow * K + first + (threadIdx.x & 15) * 128;
             for (int j = 0; j < prefetch_steps; ++j) {
-                const int64_t off = (int64_t)j * 2048 + (threadIdx.x & 15) * 128;
+                const int64_t off = first + (int64_t)j * 2048 + (threadIdx.x & 15) * 128;
                 if (off < K) {
                     sm100::prefetch_l2(P + pbase + (int64_t)j * 2048);
                     if (FULL) sm100::prefetch_l2(Rp + pbase + (int64_t)j * 2048);
@@ -91,7 +93,6 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
             }
         }
     }
-    sm100::grid_dependency_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     constexpr int kRows = HALF ? 8 : kRowsPerBlock;
@@ -166,6 +167,9 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
                     if (!HALF) wr_hi[u] = ldg_stream(r_hi + base + u * kRoundK);
                 }
             }
+            // Everything but the planes may come from the preceding kernel: wait for it here, with the
+            // first batch of weight loads already in flight.
+            if (r0 == 0) sm100::grid_dependency_wait();
             // the activation fragments of the batch are fetched together with the weights, so that
             // their (L1 / L2) latency hides behind the DRAM latency of the weight loads
             uint4 xb[U][NT][2];
@@ -179,6 +183,7 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
         // keeps the predicated copy of the loop body free of register spills), never one round at
         // a time -- a lone round costs a full DRAM latency.
         constexpr int UT = FULL ? 2 : (U > 4 ? 4 : U);
+        if (r0 == 0) sm100::grid_dependency_wait();   // K shorter than one full batch: nothing was loaded ahead
         for (; r0 < total_rounds; r0 += UT) {
             uint4 wp_lo[UT], wp_hi[UT], wr_lo[UT], wr_hi[UT];
             uint4 xb[UT][NT][2];

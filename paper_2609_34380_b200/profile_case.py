@@ -42,6 +42,7 @@ def main() -> None:
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     n, k = SHAPES[args.family][args.layer]
+    n = args.rows or n          # --rows overrides the layer's output rows (dense case too)
     enc_req = {"auto": dps.DPS_ENC_AUTO, "e4m3": dps.DPS_ENC_E4M3, "e5m2": dps.DPS_ENC_E5M2}[args.enc]
     mode = dps.DPS_MODE_FULL if args.mode == "full" else dps.DPS_MODE_FAST
     planes = []
