@@ -54,6 +54,11 @@ __host__ __device__ constexpr int block_k(bool full, int tn, int rb = 1) {
     if (rb == 2) return full ? 64 : DPS_RB2_FAST_BK;
     return (tn >= DPS_BK64_FROM || (full && tn <= 64)) ? 64 : 128;
 }
+// Widest tile whose split-K partial sums are pushed into a mailbox of their own; wider tiles keep
+// the shared memory for the ring and pull the partial tiles out of it afterwards.
+#ifndef DPS_PUSH_MAX_TN
+#define DPS_PUSH_MAX_TN 64
+#endif
 constexpr int kMaxAStages = 4;   // barrier array size for the A ring in tensor memory
 // Groups of 4 zip warps; group g takes K blocks g, g + G, ...  Two groups everywhere: four were
 // measured for 256-token full-mode tiles (one CTA per SM) and changed nothing -- once the stage
@@ -391,7 +396,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     // ring; peers store their partial sums straight into it, one cluster barrier later the owner
     // adds them in rank order.  TN >= 128 ("pull"): the partial tile red[token][row] overlays the
     // idle stage ring and owners read it out of their peers' memory between two cluster barriers.
-    constexpr bool kPush = TN <= 64;
+    constexpr bool kPush = TN <= DPS_PUSH_MAX_TN;
     float* red = reinterpret_cast<float*>(smem_raw + (smem_base - smem_u32(smem_raw)));
     const uint32_t mail_addr = smem_base + (uint32_t)prm.red_offset;
     const int slots = (TN + split - 1) / split;
@@ -1306,7 +1311,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     constexpr int kThreads = cta_threads(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
     constexpr int kSmemTotal = kCtasPerSm == 2 ? 111 * 1024 : 216 * 1024;
-    constexpr int kMailMax = TN <= 64 ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox, worst case
+    constexpr int kMailMax = TN <= DPS_PUSH_MAX_TN ? (TN + kMaxSplit) * kTileRows * 4 : 0;  // push-mode mailbox, worst case
     // Ring depth for a given mailbox size: whatever fits (stage s is rebuilt by zip group s % 2, so
     // odd depths work; they just give the first group one stage more).
     static const int deep_forced = [] {
