@@ -490,6 +490,56 @@ def detail_rows(dps, workloads, torch, dev, peaks):
     out["moe"] = moe
     torch.cuda.empty_cache()
 
+    # ---- residual restore beside fast-mode decode (the switch back to full mode) ----
+    # 8 copies of the four Llama-7B linears in fast mode, 8 tokens, as one graph on a compute stream;
+    # the residual planes of one copy (202 MB) restored from pinned host memory in 4 MiB chunks on
+    # a copy stream: alone, and while the decode graph replays.
+    copies = 8
+    fplanes = {name: [dps.dps_split_weights(workloads.weights(n, k, 2001 + i + 100 * c, device=dev), dps.DPS_ENC_AUTO)
+                      for c in range(copies)] for i, (name, (n, k)) in enumerate(workloads.LLAMA7B.items())}
+    xs = {name: workloads.activations(8, k, 2011 + i, device=dev) for i, (name, (n, k)) in enumerate(workloads.LLAMA7B.items())}
+    ys = {name: torch.empty((8, n), dtype=torch.float16, device=dev) for name, (n, k) in workloads.LLAMA7B.items()}
+
+    def fast_step():
+        for c in range(copies):
+            for name in workloads.LLAMA7B:
+                pp, rr, enc = fplanes[name][c]
+                dps.dps_linear(dps.DPS_MODE_FAST, enc, xs[name], pp, None, ys[name])
+    ms_alone, graph = _time_graph(torch, stream, fast_step, iters=20, warm=3)
+    resid = [fplanes[name][0][1] for name in workloads.LLAMA7B]
+    backups = [dps.dps_backup_residual(rr) for rr in resid]
+    torch.cuda.synchronize()
+    rbytes = sum(rr.numel() for rr in resid)
+    copy_stream = torch.cuda.Stream(device=dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(copy_stream)
+    for rr, hb in zip(resid, backups):
+        dps.dps_restore_residual(rr, hb, stream=copy_stream)
+    e1.record(copy_stream)
+    e1.synchronize()
+    restore_ms = e0.elapsed_time(e1)
+    # the same restore again while decode steps replay on the compute stream
+    steps_beside = []
+    for rr, hb in zip(resid, backups):
+        dps.dps_restore_residual(rr, hb, stream=copy_stream)
+    done = torch.cuda.Event()
+    done.record(copy_stream)
+    with torch.cuda.stream(stream):
+        while not done.query() and len(steps_beside) < 200:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            graph.replay()
+            b.record(stream)
+            b.synchronize()
+            steps_beside.append(a.elapsed_time(b))
+    torch.cuda.synchronize()
+    out["restore"] = {"bytes": rbytes, "chunk_bytes": 4 << 20, "restore_alone_GB/s": rbytes / (restore_ms * 1e-3) / 1e9,
+                      "ms_per_GB": restore_ms / (rbytes / 1e9),
+                      "fast_decode_step_ms_alone": ms_alone,
+                      "fast_decode_step_ms_beside_restore": statistics.median(steps_beside) if steps_beside else None,
+                      "steps_timed_beside_restore": len(steps_beside)}
+    del fplanes, xs, ys, graph, resid, backups
+
     # ---- 32-layer decoder step under the bursty schedule (config 5) ----
     layers = workloads.DECODER70_LAYERS
     shapes = workloads.DECODER70

@@ -174,6 +174,24 @@ DPS_API dps_status dps_moe_linear_static(int32_t mode, const int32_t* enc_per_ex
                                          void* cuda_stream);
 
 /*
+ * Residual backup and restore (paper: "Scheduler: Dual-Precision Execution", the restore of the
+ * lower byte before a switch back to full mode, done by a worker beside the running steps).
+ * While a layer runs in fast mode the memory of its residual plane may be lent out; the bytes then
+ * live in a host copy.  dps_backup_residual copies a residual plane to host memory,
+ * dps_restore_residual copies it back, both as a sequence of plain asynchronous copies of
+ * chunk_bytes each (0 = 4 MiB, the granularity at which a restore can yield to other copies) on
+ * cuda_stream -- normally a stream of its own, so that fast-mode dps_linear calls on another stream
+ * keep running meanwhile; they never read the residual plane.  backup_host should be page-locked
+ * (pinned) host memory: with pageable memory the copies are staged and the call blocks.  Neither
+ * call synchronises; the caller orders the switch to full mode after the restore (an event on
+ * cuda_stream).  bytes == 0 returns DPS_OK without enqueuing anything.
+ */
+DPS_API dps_status dps_backup_residual(const uint8_t* w_resid, uint8_t* backup_host, size_t bytes,
+                                       size_t chunk_bytes, void* cuda_stream);
+DPS_API dps_status dps_restore_residual(uint8_t* w_resid, const uint8_t* backup_host, size_t bytes,
+                                        size_t chunk_bytes, void* cuda_stream);
+
+/*
  * Synchronises the stream, then returns and clears the current device's status word:
  * DPS_OK, DPS_ERR_DATA (a kernel skipped a row with a bad index) or DPS_ERR_CUDA.
  */

@@ -31,6 +31,8 @@ ABI = {
     "dps_moe_linear_static": (ctypes.c_int, [_i32, ctypes.POINTER(_i32), _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64,
                                              _i64, _i32, _vp]),
     "dps_moe_workspace_bytes": (ctypes.c_size_t, [_i64, _i32, _i64]),
+    "dps_backup_residual": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t, ctypes.c_size_t, _vp]),
+    "dps_restore_residual": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t, ctypes.c_size_t, _vp]),
     "dps_stream_status": (ctypes.c_int, [_vp]),
     "dps_launch_count": (_i64, []),
     "dps_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -189,6 +191,34 @@ def dps_moe_linear_static(mode: int, enc_per_expert: Sequence[int], x: torch.Ten
                                          N, K, E, _stream(stream))
     _check(st, "dps_moe_linear_static")
     return y
+
+
+def _host_bytes(t: torch.Tensor, what: str) -> int:
+    if t.is_cuda or t.dtype != torch.uint8 or not t.is_contiguous():
+        raise ValueError(f"{what} must be a contiguous uint8 host tensor (pinned, for the copies to be asynchronous)")
+    return t.data_ptr()
+
+
+def dps_backup_residual(w_resid: torch.Tensor, backup_host: Optional[torch.Tensor] = None, chunk_bytes: int = 0,
+                        stream=None) -> torch.Tensor:
+    """Copy a residual plane to (pinned) host memory in chunks; returns the host tensor."""
+    if backup_host is None:
+        backup_host = torch.empty(w_resid.shape, dtype=torch.uint8, pin_memory=True)
+    if backup_host.numel() != w_resid.numel():
+        raise ValueError("backup_host has the wrong size")
+    st = library().dps_backup_residual(_dev(w_resid, torch.uint8, "w_resid"), _host_bytes(backup_host, "backup_host"),
+                                       w_resid.numel(), int(chunk_bytes), _stream(stream))
+    _check(st, "dps_backup_residual")
+    return backup_host
+
+
+def dps_restore_residual(w_resid: torch.Tensor, backup_host: torch.Tensor, chunk_bytes: int = 0, stream=None) -> None:
+    """Copy a residual plane back from its host copy in chunks, on `stream`, without synchronising."""
+    if backup_host.numel() != w_resid.numel():
+        raise ValueError("backup_host has the wrong size")
+    st = library().dps_restore_residual(_dev(w_resid, torch.uint8, "w_resid"), _host_bytes(backup_host, "backup_host"),
+                                        w_resid.numel(), int(chunk_bytes), _stream(stream))
+    _check(st, "dps_restore_residual")
 
 
 def dps_stream_status(stream=None) -> int:

@@ -230,6 +230,32 @@ dps_status dps_stream_status(void* cuda_stream) {
     return word == 0 ? DPS_OK : (word == (int)DPS_ERR_DATA ? DPS_ERR_DATA : DPS_ERR_CUDA);
 }
 
+namespace {
+dps_status chunked_copy(void* dst, const void* src, size_t bytes, size_t chunk, cudaMemcpyKind kind, void* cuda_stream) {
+    if (bytes == 0) return DPS_OK;
+    if (!dst || !src) return DPS_ERR_NULL;
+    if (chunk == 0) chunk = (size_t)4 << 20;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (size_t off = 0; off < bytes; off += chunk) {
+        const size_t n = bytes - off < chunk ? bytes - off : chunk;
+        if (cudaMemcpyAsync(static_cast<char*>(dst) + off, static_cast<const char*>(src) + off, n, kind, stream) !=
+            cudaSuccess)
+            return DPS_ERR_CUDA;
+    }
+    return DPS_OK;
+}
+}  // namespace
+
+dps_status dps_backup_residual(const uint8_t* w_resid, uint8_t* backup_host, size_t bytes, size_t chunk_bytes,
+                               void* cuda_stream) {
+    return chunked_copy(backup_host, w_resid, bytes, chunk_bytes, cudaMemcpyDeviceToHost, cuda_stream);
+}
+
+dps_status dps_restore_residual(uint8_t* w_resid, const uint8_t* backup_host, size_t bytes, size_t chunk_bytes,
+                                void* cuda_stream) {
+    return chunked_copy(w_resid, backup_host, bytes, chunk_bytes, cudaMemcpyHostToDevice, cuda_stream);
+}
+
 int64_t dps_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* dps_status_string(dps_status status) {
