@@ -59,3 +59,22 @@ def test_prefill_determinism():
     a = dps.dps_linear(dps.DPS_MODE_FULL, enc, x, p, r)
     b = dps.dps_linear(dps.DPS_MODE_FULL, enc, x, p, r)
     assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+@pytest.mark.parametrize("enc_req", [dps.DPS_ENC_AUTO, dps.DPS_ENC_E5M2])
+def test_persistent_kernel_ragged_shapes_every_output(enc_req):
+    """More tiles than SMs with a short last round, ragged in every direction: N = 2056 (17 row
+    tiles, the last with 8 rows), K = 1104 (a partial last K block, an odd number of blocks to halve),
+    M = 2500 (partial last token tile).  Full mode walks 170 tiles of 256 tokens, fast mode 180
+    two-row-block tiles; in both the last round is shared out as halves of K.  Every output is checked."""
+    N, K, M = 2056, 1104, 2500
+    w = workloads.weights(N, K, 611, device=DEV)
+    p, r, enc = dps.dps_split_weights(w, enc_req)
+    x = workloads.activations(M, K, 612, device=DEV)
+    for mode in MODES:
+        y = dps.dps_linear(mode, enc, x, p, r if mode else None)
+        ref = oracle.linear(mode, enc, to_np_words(x), to_np_bytes(p), to_np_bytes(r), threads=16)
+        assert_close_to_oracle(y, ref, f"ragged persistent mode={mode} enc={enc}")
+        again = dps.dps_linear(mode, enc, x, p, r if mode else None)
+        assert torch.equal(y, again)              # the pair reduction adds in a fixed order
+    assert dps.dps_stream_status() == dps.DPS_OK
