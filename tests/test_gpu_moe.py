@@ -136,3 +136,21 @@ def test_mixtral_shapes_sampled():
                 assert np.max(np.abs(got[a, cols] - ref)) <= 2e-3 * scale, (name, mode, a)
         assert dps.dps_stream_status() == dps.DPS_OK
         del p, r
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_persistent_grouped_kernel_with_short_last_round(mode):
+    """8 experts x 21 two-row-block tiles (N = 5128: the last tile has 8 rows) = 168 work items for 148
+    CTAs: the grouped launch runs on the persistent kernel and shares its last round out as halves of K
+    (K = 1040: a partial last K block).  Every output row is checked."""
+    E, N, K, T = 8, 5128, 1040, 256
+    p, r, encs = expert_planes(E, N, K, 900)
+    x = workloads.activations(T, K, 901, device=DEV)
+    tor, eor = workloads.top2_routing(T, E, 902)
+    args = (mode, encs, x, torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV), p, r if mode else None)
+    y = dps.dps_moe_linear(*args)
+    ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r), threads=16)
+    assert rc == oracle.OK
+    assert_close_to_oracle(y, ref, "grouped persistent")
+    assert torch.equal(y, dps.dps_moe_linear(*args))
+    assert dps.dps_stream_status() == dps.DPS_OK
