@@ -5,22 +5,29 @@
 // residual tensor into the original FP16 values *during computation*; fast mode uses the FP8
 // tensor alone.  Here that combination happens on the way from shared memory to tensor memory.
 //
-// Tile: 128 weight rows (UMMA M) x TN tokens (UMMA N), K walked in blocks of 128.  The problem
+// Tile: 128 weight rows (UMMA M) x TN tokens (UMMA N), K walked in blocks of 128 or 64.  The problem
 // is "swapped": D[row][token] = sum_k W[row][k] * x[token][k], so that even a handful of decode
 // tokens fills the 128-lane datapath with weight rows and every weight byte is fetched once.
 //
-// Roles (6 warps):
-//   warp 0     TMA producer: P tile (128 x 128 bytes), R tile (full mode), x tile (TN x 128 halves)
-//              into a ring of shared-memory stages, completion counted on mbarriers.
-//   warp 1     allocates tensor memory; one lane issues tcgen05.mma (A from TMEM, B from smem)
-//              and commits stage-release barriers.
-//   warps 2-5  "zip" warps: each owns 32 TMEM lanes = 32 weight rows.  Per K block a thread
-//              reads its row's 128 plane bytes (swizzled, conflict-free), rebuilds 128 FP16 words
-//              in registers with byte permutes and writes them to the A ring in TMEM with one
-//              tcgen05.st.  After the K loop the same warps drain the accumulator
-//              (tcgen05.ld), round to FP16 and store y.
+// Roles (10 warps):
+//   warp 0     TMA producer: P tile (128 rows x 128 or 64 bytes), R tile (full mode), x tile (TN rows
+//              of 64-element swizzle atoms) into a ring of shared-memory stages, completion
+//              counted on mbarriers.  32-token tiles keep x in three slots of their own.
+//   warp 1     allocates tensor memory; one elected lane issues tcgen05.mma (A from TMEM, B from
+//              smem) and commits stage-release barriers.
+//   warps 2-9  two groups of four "zip" warps; a warp owns 32 TMEM lanes = 32 weight rows.  Per K
+//              block a thread reads its row's plane bytes (swizzled, conflict-free), rebuilds the
+//              FP16 words in registers (byte permutes; hardware FP8 conversion for E4M3 fast mode)
+//              and writes them to the A ring in TMEM with tcgen05.st.  The groups alternate K
+//              blocks, or (RB = 2) serve one 128-row block each of a 256-row CTA tile.  After the
+//              K loop the zip warps drain the accumulator (tcgen05.ld), round to FP16 and store y
+//              through a shared-memory tile with 16-byte stores.
 // Shared memory never holds FP16 weights, so its bandwidth is spent on 1-2 bytes per weight
 // instead of 5-6, and the tensor core reads only the small activation tile from it.
+//
+// Two kernels share these roles: umma_linear_kernel (one tile per CTA; K split over a cluster with
+// a DSMEM mailbox for decode-sized tiles) and umma_persistent_kernel (one CTA per SM walks many tiles;
+// prefill and grouped launches), see below.
 #include <cuda_fp16.h>
 
 #include <cstdio>
