@@ -1,4 +1,5 @@
-// Decode linear layer for up to 16 tokens: a register-streaming kernel.
+// Decode linear layer for a handful of tokens (up to 16; NT = 4 for up to 32 exists for comparison):
+// a register-streaming kernel.
 //
 // Paper: "Scheduler: Dual-Precision Execution" -- fast mode streams the FP8 tensor only, full mode
 // streams the FP8 and the residual tensor and rebuilds the FP16 weights during computation.  With
@@ -15,7 +16,10 @@
 //   * the K order inside an MMA is free as long as both operands agree, which is what lets each
 //     lane feed 16 consecutive bytes of one row (four MMAs' worth) without any shuffle;
 //   * partial sums of the eight warps are added in a fixed order through shared memory, so the
-//     result is bit-stable.  CTAs walk the 16-row blocks of the matrix persistently.
+//     result is bit-stable.  One CTA per 16-row block: the hardware scheduler balances the SMs;
+//   * the first batch of weight loads is issued before the kernel waits for its predecessor in
+//     the stream (programmatic dependent launch): the planes are model state, only the
+//     activations can be that predecessor's output.
 // Tensor memory and TMA buy nothing here (no reuse, nothing to stage); the wide tcgen05 tiles take
 // over once the token count makes the layer a real contraction.
 #include <cuda_fp16.h>
