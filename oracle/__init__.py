@@ -72,6 +72,14 @@ def lib() -> ctypes.CDLL:
         L.oracle_moe_linear.restype = ctypes.c_int
         L.oracle_moe_linear.argtypes = [ctypes.c_int, vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64,
                                         i64, i32, vp, i64, ctypes.c_int]
+        L.oracle_e4m3_to_double.restype = ctypes.c_double
+        L.oracle_e4m3_to_double.argtypes = [ctypes.c_uint8]
+        L.oracle_float_to_e4m3.restype = ctypes.c_uint8
+        L.oracle_float_to_e4m3.argtypes = [ctypes.c_float]
+        L.oracle_quantize_activations.restype = ctypes.c_int
+        L.oracle_quantize_activations.argtypes = [vp, vp, vp, i64, i64]
+        L.oracle_linear_fp8act.restype = ctypes.c_int
+        L.oracle_linear_fp8act.argtypes = [ctypes.c_int, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int]
         _lib = L
     return _lib
 
@@ -189,6 +197,40 @@ def linear_at(mode: int, enc: int, x, p, r, ms, ns) -> np.ndarray:
     if rc != OK:
         raise OracleError(rc, "linear_at")
     return out
+
+
+def e4m3_to_double(code: int) -> float:
+    return float(lib().oracle_e4m3_to_double(int(code) & 0xFF))
+
+
+def float_to_e4m3(v: float) -> int:
+    """binary32 value -> E4M3 code, round to nearest even, saturating at +-448."""
+    return int(lib().oracle_float_to_e4m3(float(np.float32(v))))
+
+
+def quantize_activations(x):
+    """FP16 words [M][K] -> (E4M3 codes uint8 [M][K], per-token scale float32 [M])."""
+    x = _words(x)
+    M, K = x.shape
+    q = np.empty((M, K), np.uint8)
+    scale = np.empty((M,), np.float32)
+    rc = lib().oracle_quantize_activations(_ptr(x), _ptr(q), _ptr(scale), M, K)
+    if rc != OK:
+        raise OracleError(rc, "quantize_activations")
+    return q, scale
+
+
+def linear_fp8act(enc: int, q, scale, p, threads: int = 1) -> np.ndarray:
+    """Fast-mode linear with FP8 activations: y_ref[m][n] = scale[m] * sum_k e4m3(q[m][k]) * W_fast[n][k] (float64)."""
+    q, p = _bytes(q), _bytes(p)
+    scale = np.ascontiguousarray(scale, np.float32)
+    M, K = q.shape
+    N, _ = p.shape
+    y = np.zeros((M, N), np.float64)
+    rc = lib().oracle_linear_fp8act(enc, _ptr(q), _ptr(scale), _ptr(p), _ptr(y), M, N, K, int(threads))
+    if rc != OK:
+        raise OracleError(rc, "linear_fp8act")
+    return y
 
 
 def moe_linear(mode: int, enc_per_expert, x, token_of_row, expert_of_row, p, r, rows=None,

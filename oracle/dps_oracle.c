@@ -256,4 +256,92 @@ int oracle_moe_linear(int mode, const int32_t* enc_per_expert, const uint16_t* x
     return bad ? ORACLE_ERR_DATA : ORACLE_OK;
 }
 
-int oracle_version(void) { return 1; }
+/* ---- FP8 activations for fast mode (the paper's "doubling peak tensor-core throughput with
+ * hardware support" option: "Persistent Region" paragraph, remark on FP8 execution).  The paper
+ * gives no recipe; the reading taken (listed in the design notes) is per-token dynamic scaling:
+ *   scale[m] = max_k |x[m][k]| / 448   (448 = largest finite E4M3 value; 1 if the row is all zero),
+ *   q[m][k]  = E4M3( x[m][k] / scale[m] ), round to nearest even, saturating,
+ * both computed in binary32 (the precision the decision is taken in), and
+ *   y_ref[m][n] = scale[m] * sum_k value(q[m][k]) * W_fast[n][k]   in FP64.
+ * E4M3 here is the 8-bit format with bias 7, no infinities, one NaN code per sign (0x7F / 0xFF),
+ * subnormals with exponent field 0: value = (-1)^s 2^(e-7) (1 + m/8), or 2^-6 (m/8) for e = 0. */
+
+double oracle_e4m3_to_double(uint8_t b) {
+    int s = b >> 7, e = (b >> 3) & 0xF, m = b & 7;
+    double v;
+    if (e == 0xF && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m / 8.0, -6);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return s ? -v : v;
+}
+
+/* binary32 -> E4M3, round to nearest even, values beyond 448 saturate to +-448, NaN -> 0x7F.
+ * Written from the format: find the two neighbouring representable values and pick the nearer,
+ * the one with even mantissa code on a tie. */
+uint8_t oracle_float_to_e4m3(float f) {
+    if (f != f) return 0x7F;
+    uint8_t sign = (f < 0.0f || (f == 0.0f && 1.0f / f < 0.0f)) ? 0x80 : 0x00;
+    double a = fabs((double)f);
+    if (a >= 448.0) return sign | 0x7E;
+    /* codes 0x00..0x7E are monotone in value: binary search for the largest code with value <= a */
+    int lo = 0, hi = 0x7E;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) / 2;
+        if (oracle_e4m3_to_double((uint8_t)mid) <= a) lo = mid; else hi = mid - 1;
+    }
+    if (lo < 0x7E) {
+        double below = oracle_e4m3_to_double((uint8_t)lo), above = oracle_e4m3_to_double((uint8_t)(lo + 1));
+        double d0 = a - below, d1 = above - a;
+        if (d1 < d0 || (d1 == d0 && (lo & 1))) lo += 1;
+    }
+    return sign | (uint8_t)lo;
+}
+
+/* x: FP16 words [M][K] -> q: E4M3 bytes [M][K], scale: binary32 [M]. */
+int oracle_quantize_activations(const uint16_t* x, uint8_t* q, float* scale, int64_t M, int64_t K) {
+    for (int64_t m = 0; m < M; ++m) {
+        float amax = 0.0f;
+        for (int64_t k = 0; k < K; ++k) {
+            float v = (float)fabs(oracle_half_to_double(x[m * K + k]));
+            if (v != v) return ORACLE_ERR_DATA;
+            if (v > amax) amax = v;
+        }
+        if (isinf(amax)) return ORACLE_ERR_DATA;
+        float sc = amax > 0.0f ? amax / 448.0f : 1.0f;   /* binary32 division, round to nearest */
+        scale[m] = sc;
+        for (int64_t k = 0; k < K; ++k) {
+            float v = (float)oracle_half_to_double(x[m * K + k]);
+            q[m * K + k] = oracle_float_to_e4m3(v / sc);   /* binary32 division, then one rounding to E4M3 */
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* y_ref[m][n] = scale[m] * sum_k value(q[m][k]) * W_fast[n][k], FP64, k ascending. */
+int oracle_linear_fp8act(int enc, const uint8_t* q, const float* scale, const uint8_t* p, double* y_ref, int64_t M,
+                         int64_t N, int64_t K, int threads) {
+    if (enc != ORACLE_ENC_E4M3 && enc != ORACLE_ENC_E5M2) return ORACLE_ERR_ARG;
+    if (M == 0 || N == 0) return ORACLE_OK;
+    double* xd = (double*)malloc(sizeof(double) * (size_t)(M * K > 0 ? M * K : 1));
+    if (!xd) return ORACLE_ERR_ARG;
+    for (int64_t i = 0; i < M * K; ++i) xd[i] = oracle_e4m3_to_double(q[i]);
+    if (threads < 1) threads = 1;
+#pragma omp parallel num_threads(threads)
+    {
+        double* wrow = (double*)malloc(sizeof(double) * (size_t)(K > 0 ? K : 1));
+#pragma omp for schedule(static)
+        for (int64_t n = 0; n < N; ++n) {
+            for (int64_t k = 0; k < K; ++k) wrow[k] = eff_weight(ORACLE_MODE_FAST, enc, p, NULL, n * K + k);
+            for (int64_t m = 0; m < M; ++m) {
+                double acc = 0.0;
+                for (int64_t k = 0; k < K; ++k) acc += xd[m * K + k] * wrow[k];
+                y_ref[m * N + n] = acc * (double)scale[m];
+            }
+        }
+        free(wrow);
+    }
+    free(xd);
+    return ORACLE_OK;
+}
+
+int oracle_version(void) { return 2; }
