@@ -174,6 +174,26 @@ DPS_API dps_status dps_moe_linear_static(int32_t mode, const int32_t* enc_per_ex
                                          void* cuda_stream);
 
 /*
+ * Fast mode with FP8 activations (paper: "Persistent Region" paragraph -- FP8 execution can "double
+ * peak tensor-core throughput with hardware support").  The persistent plane is fed to the FP8
+ * tensor cores as it is; the activations are quantised per token:
+ *   scale[m] = max_k |x[m][k]| / 448 (1 for an all-zero token),
+ *   x_fp8[m][k] = E4M3(x[m][k] / scale[m]), round to nearest even, saturating (both in binary32),
+ *   y[m][n] = scale[m] * sum_k x_fp8[m][k] * W_fast[n][k], FP32 accumulation, one FP16 rounding.
+ * This is a DIFFERENT result from dps_linear in fast mode (the activations lose precision: a few
+ * per cent of the output scale on Gaussian data); it is meant for prefill-sized token counts.
+ * dps_quantize_activations: x FP16 [M][K] -> x_fp8 uint8 [M][K] and scale float [M] (all device).
+ * An Inf or NaN activation sets the device status word to DPS_ERR_DATA.
+ * dps_linear_fp8act: enc as reported by dps_split_weights; the residual plane is not an argument.
+ * Shapes, alignment and error rules as for dps_linear.  Neither call synchronises or allocates.
+ */
+DPS_API dps_status dps_quantize_activations(const void* x, uint8_t* x_fp8, float* scale, int64_t M, int64_t K,
+                                            void* cuda_stream);
+DPS_API dps_status dps_linear_fp8act(int32_t enc, const uint8_t* x_fp8, const float* scale,
+                                     const uint8_t* w_persist, void* y, int64_t M, int64_t N, int64_t K,
+                                     void* cuda_stream);
+
+/*
  * Residual backup and restore (paper: "Scheduler: Dual-Precision Execution", the restore of the
  * lower byte before a switch back to full mode, done by a worker beside the running steps).
  * While a layer runs in fast mode the memory of its residual plane may be lent out; the bytes then

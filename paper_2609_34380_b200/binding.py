@@ -31,6 +31,8 @@ ABI = {
     "dps_moe_linear_static": (ctypes.c_int, [_i32, ctypes.POINTER(_i32), _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64,
                                              _i64, _i32, _vp]),
     "dps_moe_workspace_bytes": (ctypes.c_size_t, [_i64, _i32, _i64]),
+    "dps_quantize_activations": (ctypes.c_int, [_vp, _vp, _vp, _i64, _i64, _vp]),
+    "dps_linear_fp8act": (ctypes.c_int, [_i32, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp]),
     "dps_backup_residual": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t, ctypes.c_size_t, _vp]),
     "dps_restore_residual": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t, ctypes.c_size_t, _vp]),
     "dps_stream_status": (ctypes.c_int, [_vp]),
@@ -190,6 +192,36 @@ def dps_moe_linear_static(mode: int, enc_per_expert: Sequence[int], x: torch.Ten
                                          _dev(w_resid, torch.uint8, "w_resid"), _dev(y, torch.float16, "y"), A, T,
                                          N, K, E, _stream(stream))
     _check(st, "dps_moe_linear_static")
+    return y
+
+
+def dps_quantize_activations(x: torch.Tensor, x_fp8: Optional[torch.Tensor] = None,
+                             scale: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """FP16 x[M][K] -> (E4M3 codes uint8 [M][K], per-token scale float32 [M])."""
+    M, K = x.shape
+    if x_fp8 is None:
+        x_fp8 = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+    if scale is None:
+        scale = torch.empty((M,), dtype=torch.float32, device=x.device)
+    st = library().dps_quantize_activations(_dev(x, torch.float16, "x"), _dev(x_fp8, torch.uint8, "x_fp8"),
+                                            _dev(scale, torch.float32, "scale"), M, K, _stream(stream))
+    _check(st, "dps_quantize_activations")
+    return x_fp8, scale
+
+
+def dps_linear_fp8act(enc: int, x_fp8: torch.Tensor, scale: torch.Tensor, w_persist: torch.Tensor,
+                      y: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Fast mode with FP8 activations: y[M][N] = scale[m] * x_fp8 * W_fast^T on the FP8 tensor cores."""
+    M, K = x_fp8.shape
+    N, K2 = w_persist.shape
+    if K != K2:
+        raise ValueError(f"K mismatch: x_fp8 has {K}, the plane has {K2}")
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float16, device=x_fp8.device)
+    st = library().dps_linear_fp8act(int(enc), _dev(x_fp8, torch.uint8, "x_fp8"), _dev(scale, torch.float32, "scale"),
+                                     _dev(w_persist, torch.uint8, "w_persist"), _dev(y, torch.float16, "y"), M, N, K,
+                                     _stream(stream))
+    _check(st, "dps_linear_fp8act")
     return y
 
 

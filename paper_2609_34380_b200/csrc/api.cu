@@ -230,6 +230,38 @@ dps_status dps_stream_status(void* cuda_stream) {
     return word == 0 ? DPS_OK : (word == (int)DPS_ERR_DATA ? DPS_ERR_DATA : DPS_ERR_CUDA);
 }
 
+dps_status dps_quantize_activations(const void* x, uint8_t* x_fp8, float* scale, int64_t M, int64_t K,
+                                    void* cuda_stream) {
+    if (M < 0 || K <= 0 || (K % 16) != 0 || M > ((int64_t)1 << 31) || K > ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
+    if (M == 0) return DPS_OK;
+    if (!x || !x_fp8 || !scale) return DPS_ERR_NULL;
+    if (!aligned16(x) || !aligned16(x_fp8)) return DPS_ERR_ALIGN;
+    DeviceInfo* d;
+    dps_status st = check_device(d);
+    if (st != DPS_OK) return st;
+    return launch_quantize_activations(x, x_fp8, scale, M, K, d->status, static_cast<cudaStream_t>(cuda_stream)) ==
+                   cudaSuccess
+               ? DPS_OK
+               : DPS_ERR_CUDA;
+}
+
+dps_status dps_linear_fp8act(int32_t enc, const uint8_t* x_fp8, const float* scale, const uint8_t* w_persist, void* y,
+                             int64_t M, int64_t N, int64_t K, void* cuda_stream) {
+    if (enc != DPS_ENC_E4M3 && enc != DPS_ENC_E5M2) return DPS_ERR_ENCODING;
+    if (M < 0 || N <= 0 || K <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
+    if (N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31) || M > ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
+    if (M == 0) return DPS_OK;
+    if (!x_fp8 || !scale || !w_persist || !y) return DPS_ERR_NULL;
+    if (!aligned16(x_fp8) || !aligned16(w_persist) || !aligned16(y)) return DPS_ERR_ALIGN;
+    DeviceInfo* d;
+    dps_status st = check_device(d);
+    if (st != DPS_OK) return st;
+    return launch_linear_fp8act(enc, x_fp8, scale, w_persist, y, M, N, K, d->status,
+                                static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? DPS_OK
+               : DPS_ERR_CUDA;
+}
+
 namespace {
 dps_status chunked_copy(void* dst, const void* src, size_t bytes, size_t chunk, cudaMemcpyKind kind, void* cuda_stream) {
     if (bytes == 0) return DPS_OK;

@@ -39,6 +39,13 @@ cudaError_t launch_umma_grouped(int mode, const uint32_t* e5m2_mask, const void*
                                 const void* tiles, const int32_t* num_tiles, const int32_t* sorted_rows,
                                 int max_tiles, int* status, cudaStream_t stream);
 
+// Fast mode with FP8 activations: per-token E4M3 quantisation, then an FP8 x FP8 tensor-core linear
+// that reads the persistent plane as it is.
+cudaError_t launch_quantize_activations(const void* x, uint8_t* q, float* scale, int64_t M, int64_t K, int* status,
+                                        cudaStream_t stream);
+cudaError_t launch_linear_fp8act(int enc, const uint8_t* q, const float* scale, const uint8_t* p, void* y, int64_t M,
+                                 int64_t N, int64_t K, int* status, cudaStream_t stream);
+
 // Grouped linear.
 size_t moe_workspace_bytes(int64_t A, int32_t E, int64_t K);
 cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const int32_t* token_of_row,

@@ -1570,6 +1570,12 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
 
 }  // namespace
 
+// Byte-matrix tensor map for the other translation units (row-major [rows][cols] bytes, boxes of
+// box_rows x 128 bytes, 128-byte swizzle).
+bool make_byte_map_sw128(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    return make_map_2d(map, base, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, rows, cols, box_rows, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
 #ifdef DPS_TRACE
 extern "C" __attribute__((visibility("default"))) int dps_debug_trace(long long* out, int max_words) {
     const int n = max_words < kTraceBlocks * kTraceEvents ? max_words : kTraceBlocks * kTraceEvents;
