@@ -454,6 +454,23 @@ def detail_rows(dps, workloads, torch, dev, peaks):
             pre[f"M{M}_{'full' if mode else 'fast'}"] = {"TFLOP/s": tf, "frac_of_measured_bf16_burst": tf / tc,
                                                         "frac_of_measured_bf16_sustained": tf / peaks["bf16_tflops_sustained"],
                                                         "ms_per_layer_set": ms / 4}
+            if mode == dps.DPS_MODE_FAST:
+                # the same layer set in fast mode with FP8 activations: quantisation + FP8 x FP8 linears
+                qs = {name: dps.dps_quantize_activations(xs[name]) for name in workloads.LLAMA7B}
+
+                def enqueue_fp8():
+                    for c in range(4):
+                        for name in workloads.LLAMA7B:
+                            p, r, enc = planes[name][c]
+                            dps.dps_quantize_activations(xs[name], qs[name][0], qs[name][1])
+                            dps.dps_linear_fp8act(enc, qs[name][0], qs[name][1], p, ys[name])
+                ms8, _ = _time_graph(torch, stream, enqueue_fp8, iters=3, warm=1)
+                tf8 = flops / (ms8 * 1e-3) / 1e12
+                # FP8 dense peak: the measured BF16 figures times the nominal FP8 : BF16 ratio of 2
+                pre[f"M{M}_fast_fp8act"] = {"TFLOP/s": tf8, "frac_of_2x_measured_bf16_burst": tf8 / (2 * tc),
+                                            "frac_of_2x_measured_bf16_sustained": tf8 / (2 * peaks["bf16_tflops_sustained"]),
+                                            "ms_per_layer_set": ms8 / 4, "includes": "per-token activation quantisation"}
+                del qs
         del xs, ys
     out["prefill"] = pre
     del planes
