@@ -11,9 +11,10 @@
 // taken): scale[m] = max_k |x[m][k]| / 448 (1 for an all-zero token), q = E4M3(x / scale), round to
 // nearest even, saturating; y[m][n] = scale[m] * sum_k q[m][k] * W_fast[n][k].
 //
-// Kernel: 128 weight rows x 256 tokens per CTA, K in blocks of 128 bytes.  Warp 0 TMA producer
-// (P tile 128 x 128 B, activation tile 256 x 128 B, 128-byte swizzle), warp 1 MMA issuer, warps 2-5
-// epilogue (TMEM -> scale -> FP16 -> shared-memory tile -> 16-byte stores).
+// Kernel: tiles of 128 weight rows x 256 tokens, K in blocks of 128 bytes, one persistent CTA per
+// SM.  Warp 0 TMA producer (P tile 128 x 128 B, activation tile 256 x 128 B, 128-byte swizzle), warp 1
+// MMA issuer (two accumulators in tensor memory), warps 2-5 epilogue (TMEM -> scale -> FP16 ->
+// shared-memory buffer -> 16-byte stores), overlapped with the next tile's MMAs.
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
@@ -91,7 +92,7 @@ constexpr int kBlockBytes = 128;                                  // K per stage
 constexpr int kStageBytes = (kRows + kTokens) * kBlockBytes;      // 48 KB
 constexpr int kStages = 4;
 constexpr int kThreads = 192;
-constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kTmemCols = 512;   // two accumulators of 256 token columns
 
 // Instruction descriptor for kind::f8f6f4: FP32 accumulator, K-major operands; formats 0 = E4M3, 1 = E5M2.
 __host__ __device__ constexpr uint32_t idesc_f8(int m, int n, int a_format, int b_format) {
@@ -118,38 +119,56 @@ struct Fp8Params {
     int* status;
 };
 
+constexpr int kEpiCols = 32;                                      // token columns per epilogue chunk
+constexpr int kEpiBytes = kEpiCols * kRows * 2;                   // 8 KB buffer behind the ring
+
+// Persistent: one CTA per SM walks the tiles (groups of 8 row tiles x all token tiles).  Two
+// accumulators of 256 columns fill tensor memory, so the MMA warp starts the next tile while the
+// four epilogue warps drain the previous one -- at FP8 rates the epilogue of a 128 x 256 tile is a
+// fifth of the tile's MMA time.  The epilogue goes through a small buffer, 32 token columns at a
+// time: the stage ring never idles.
 __global__ void __launch_bounds__(kThreads, 1)
 fp8act_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_x,
                      const Fp8Params prm) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[kStages];
     __shared__ __align__(8) uint64_t bar_empty[kStages];
-    __shared__ __align__(8) uint64_t bar_d_full;
+    __shared__ __align__(8) uint64_t bar_d_full[2];
+    __shared__ __align__(8) uint64_t bar_d_empty[2];
     __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;    // set by an epilogue warp whose wait timed out; the four leave together
 
     grid_launch_dependents();
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t epi_base = smem_base + (uint32_t)(kStages * kStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // groups of 8 row tiles x all token tiles, as in the FP16-activation kernel (L2 reuse of planes and activations)
-    int row_tile = blockIdx.x, tok_tile = blockIdx.y;
-    if (gridDim.y > 1) {
-        constexpr int kRowGroup = 8;
-        const int lin = blockIdx.x + gridDim.x * blockIdx.y;
-        const int per_group = kRowGroup * gridDim.y;
-        const int group = lin / per_group, within = lin % per_group;
-        const int rows_here = min(kRowGroup, (int)gridDim.x - group * kRowGroup);
-        row_tile = group * kRowGroup + within % rows_here;
-        tok_tile = within / rows_here;
-    }
-    const int n0 = row_tile * kRows, m0 = tok_tile * kTokens;
+    const int row_tiles = (prm.N + kRows - 1) / kRows, tok_tiles = (prm.M + kTokens - 1) / kTokens;
+    const int total = row_tiles * tok_tiles;
     const int num_kb = (prm.K + kBlockBytes - 1) / kBlockBytes;
+    auto tile_origin = [&](int lin, int& n0, int& m0) {
+        int row_tile = lin, tok_tile = 0;
+        if (tok_tiles > 1) {
+            constexpr int kRowGroup = 8;
+            const int per_group = kRowGroup * tok_tiles;
+            const int group = lin / per_group, within = lin % per_group;
+            const int rows_here = min(kRowGroup, row_tiles - group * kRowGroup);
+            row_tile = group * kRowGroup + within % rows_here;
+            tok_tile = within / rows_here;
+        }
+        n0 = row_tile * kRows;
+        m0 = tok_tile * kTokens;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
             mbar_init(smem_u32(&bar_empty[s]), 1);
         }
-        mbar_init(smem_u32(&bar_d_full), 1);
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&bar_d_full[a]), 1);
+            mbar_init(smem_u32(&bar_d_empty[a]), 4);   // one arrival per epilogue warp
+        }
+        abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_p);
         prefetch_tensormap(&map_x);
@@ -158,7 +177,7 @@ fp8act_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem_d = tmem_base_slot;
+    const uint32_t tmem_base = tmem_base_slot;
 
     bool ok = true;
     if (warp == 0) {
@@ -166,40 +185,54 @@ fp8act_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
         grid_dependency_wait();   // the activation codes come from the quantisation kernel
         int s = 0;
         uint32_t ph = 0;
-        for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == kStages) ? 0 : s + 1, ph ^= (s == 0)) {
-            ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            if (elect_one()) {
-                const uint32_t full = smem_u32(&bar_full[s]);
-                const uint32_t dst = smem_base + (uint32_t)s * kStageBytes;
-                mbar_arrive_expect_tx(full, (uint32_t)kStageBytes);
-                tma_load_2d(dst, &map_p, full, i * kBlockBytes, n0);
-                tma_load_2d(dst + kRows * kBlockBytes, &map_x, full, i * kBlockBytes, m0);
+        for (int lin = blockIdx.x; lin < total && ok; lin += gridDim.x) {
+            int n0, m0;
+            tile_origin(lin, n0, m0);
+            for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == kStages) ? 0 : s + 1, ph ^= (s == 0)) {
+                ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                if (elect_one()) {
+                    const uint32_t full = smem_u32(&bar_full[s]);
+                    const uint32_t dst = smem_base + (uint32_t)s * kStageBytes;
+                    mbar_arrive_expect_tx(full, (uint32_t)kStageBytes);
+                    tma_load_2d(dst, &map_p, full, i * kBlockBytes, n0);
+                    tma_load_2d(dst + kRows * kBlockBytes, &map_x, full, i * kBlockBytes, m0);
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         const uint32_t idesc = idesc_f8(kRows, kTokens, prm.e5m2 ? 1 : 0, 0);
-        int s = 0;
+        int s = 0, it = 0;
         uint32_t ph = 0;
-        for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == kStages) ? 0 : s + 1, ph ^= (s == 0)) {
-            ok = mbar_wait(smem_u32(&bar_full[s]), ph);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            tc_fence_after_sync();
-            if (elect_one()) {
-                const uint32_t abase = smem_base + (uint32_t)s * kStageBytes;
-                const uint64_t adesc = umma_desc_k_sw128(abase), bdesc = umma_desc_k_sw128(abase + kRows * kBlockBytes);
-#pragma unroll
-                for (int j = 0; j < kBlockBytes / 32; ++j)   // 32 K elements = 32 bytes per instruction
-                    umma_f8_ss(tmem_d, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc,
-                               (i > 0 || j > 0) ? 1u : 0u);
-                umma_commit(smem_u32(&bar_empty[s]));
-                if (i == num_kb - 1) umma_commit(smem_u32(&bar_d_full));
+        for (int lin = blockIdx.x; lin < total && ok; lin += gridDim.x, ++it) {
+            const int acc = it & 1;
+            if (it >= 2) {   // the tile before last used this accumulator: its epilogue must have read it out
+                ok = mbar_wait(smem_u32(&bar_d_empty[acc]), (uint32_t)((it >> 1) - 1) & 1u);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
             }
-            __syncwarp();
+            const uint32_t tmem_d = tmem_base + (uint32_t)(acc * kTokens);
+            for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == kStages) ? 0 : s + 1, ph ^= (s == 0)) {
+                ok = mbar_wait(smem_u32(&bar_full[s]), ph);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (elect_one()) {
+                    const uint32_t abase = smem_base + (uint32_t)s * kStageBytes;
+                    const uint64_t adesc = umma_desc_k_sw128(abase), bdesc = umma_desc_k_sw128(abase + kRows * kBlockBytes);
+#pragma unroll
+                    for (int j = 0; j < kBlockBytes / 32; ++j)   // 32 K elements = 32 bytes per instruction
+                        umma_f8_ss(tmem_d, adesc + (uint64_t)(j * 2), bdesc + (uint64_t)(j * 2), idesc,
+                                   (i > 0 || j > 0) ? 1u : 0u);
+                    umma_commit(smem_u32(&bar_empty[s]));
+                    if (i == num_kb - 1) umma_commit(smem_u32(&bar_d_full[acc]));
+                }
+                __syncwarp();
+            }
         }
     } else {
         // ---------------- epilogue: D[row][token] * scale[token] -> FP16 -> y[token][n0 + row] ----------------
@@ -207,38 +240,63 @@ fp8act_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
         const int row = q * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const float wscale = prm.e5m2 ? 1.0f : 0.00390625f;   // E4M3 bytes read as FP8 are 2^8 times the weights
-        const int ncols = min(kTokens, prm.M - m0);
-        ok = mbar_wait(smem_u32(&bar_d_full), 0u);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (ok) {
-            tc_fence_after_sync();
-            for (int c0 = 0; c0 < ncols; c0 += 16) {
-                uint32_t v[16];
-                tmem_ld_32x32b_x16(tmem_d + lane_base + (uint32_t)c0, v);
-                tmem_wait_ld();
+        const int et = (int)threadIdx.x - 64;            // index among the 128 epilogue threads
+        int it = 0;
+        for (int lin = blockIdx.x; lin < total; lin += gridDim.x, ++it) {
+            int n0, m0;
+            tile_origin(lin, n0, m0);
+            const int acc = it & 1;
+            const uint32_t tmem_d = tmem_base + (uint32_t)(acc * kTokens);
+            const int ncols = min(kTokens, prm.M - m0);
+            if (ok) ok = mbar_wait(smem_u32(&bar_d_full[acc]), (uint32_t)(it >> 1) & 1u);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (ok) tc_fence_after_sync();
+            else abort_flag = 1;
+            // same trip count in all four warps (it depends on the tile only): the barriers always match
+            for (int c0 = 0; c0 < ncols; c0 += kEpiCols) {
+                if (ok) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int c = c0 + j;
-                    const float sc = c < ncols ? prm.scale[m0 + c] * wscale : 0.f;
-                    const __half h = __float2half_rn(__uint_as_float(v[j]) * sc);
-                    // the tile [token][row] overlays the idle ring: every load has been consumed
-                    const uint32_t addr = smem_base + (uint32_t)((c * kRows + row) * 2);
-                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(h)) : "memory");
+                    for (int h = 0; h < kEpiCols / 16; ++h) {
+                        const int cb = c0 + 16 * h;
+                        if (cb >= ncols) break;
+                        uint32_t v[16];
+                        tmem_ld_32x32b_x16(tmem_d + lane_base + (uint32_t)cb, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int c = cb + j;
+                            const float sc = c < ncols ? prm.scale[m0 + c] * wscale : 0.f;
+                            const __half hv = __float2half_rn(__uint_as_float(v[j]) * sc);
+                            const uint32_t addr = epi_base + (uint32_t)(((c - c0) * kRows + row) * 2);
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(hv)) : "memory");
+                        }
+                    }
                 }
+                if (c0 + kEpiCols >= ncols) {            // last chunk read: the accumulator is free again
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_d_empty[acc]));
+                }
+                named_barrier_sync(1, 128);
+                if (ok) {
+                    constexpr int kChunks = kRows / 8;   // 16-byte pieces of one token's rows
+                    const int cols_here = min(kEpiCols, ncols - c0);
+                    for (int item = et; item < cols_here * kChunks; item += 128) {
+                        const int c = item / kChunks, qq = item % kChunks;
+                        const int n = n0 + qq * 8;
+                        if (n >= prm.N) continue;        // N is a multiple of 8
+                        uint4 val;
+                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                     : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
+                                     : "r"(epi_base + (uint32_t)((c * kRows + qq * 8) * 2)));
+                        *reinterpret_cast<uint4*>(prm.y + (int64_t)(m0 + c0 + c) * prm.N + n) = val;
+                    }
+                }
+                named_barrier_sync(1, 128);              // the buffer is free for the next chunk
             }
-        }
-        named_barrier_sync(1, 128);                      // the four epilogue warps
-        if (ok) {
-            constexpr int kChunks = kRows / 8;           // 16-byte pieces of one token's rows
-            for (int item = (int)threadIdx.x - 64; item < ncols * kChunks; item += 128) {
-                const int c = item / kChunks, qq = item % kChunks;
-                const int n = n0 + qq * 8;
-                if (n >= prm.N) continue;                // N is a multiple of 8
-                uint4 val;
-                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                             : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
-                             : "r"(smem_base + (uint32_t)((c * kRows + qq * 8) * 2)));
-                *reinterpret_cast<uint4*>(prm.y + (int64_t)(m0 + c) * prm.N + n) = val;
+            if (*reinterpret_cast<volatile int*>(&abort_flag)) {   // read after the tile's last barrier: the same in all four warps
+                ok = false;
+                break;
             }
         }
     }
@@ -247,7 +305,7 @@ fp8act_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_con
     __syncthreads();
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_d, kTmemCols);
+        tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -273,7 +331,7 @@ cudaError_t launch_quantize_activations(const void* x, uint8_t* q, float* scale,
 cudaError_t launch_linear_fp8act(int enc, const uint8_t* q, const float* scale, const uint8_t* p, void* y, int64_t M,
                                  int64_t N, int64_t K, int* status, cudaStream_t stream) {
     static bool configured = false;
-    const size_t smem = (size_t)kStages * kStageBytes + 1024;
+    const size_t smem = (size_t)kStages * kStageBytes + kEpiBytes + 1024;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(fp8act_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -291,8 +349,9 @@ cudaError_t launch_linear_fp8act(int enc, const uint8_t* q, const float* scale, 
     prm.K = (int)K;
     prm.e5m2 = enc == DPS_ENC_E5M2;
     prm.status = status;
+    const int64_t tiles = ((N + kRows - 1) / kRows) * ((M + kTokens - 1) / kTokens);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)((N + kRows - 1) / kRows), (unsigned)((M + kTokens - 1) / kTokens), 1);
+    cfg.gridDim = dim3((unsigned)(tiles < sm_count() ? tiles : sm_count()), 1, 1);   // one CTA per SM walks the tiles
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
