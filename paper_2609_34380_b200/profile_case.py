@@ -33,6 +33,7 @@ def main() -> None:
     ap.add_argument("--enc", default="auto", choices=["auto", "e4m3", "e5m2"])
     ap.add_argument("--copies", type=int, default=4)
     ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--fp8act", action="store_true", help="fast mode with FP8 activations (quantisation + FP8 linear)")
     ap.add_argument("--experts", type=int, default=0, help="> 0: grouped (MoE) linear over this many experts")
     ap.add_argument("--rows", type=int, default=0, help="grouped case: output rows per expert (0 = the layer's)")
     args = ap.parse_args()
@@ -52,9 +53,16 @@ def main() -> None:
         del w
     x = workloads.activations(args.M, k, 2011, device=dev)
     y = torch.empty((args.M, n), dtype=torch.float16, device=dev)
+    if args.fp8act:
+        q, scale = dps.dps_quantize_activations(x)
+
     def enqueue():
         for p, r, enc in planes:
-            dps.dps_linear(mode, enc, x, p, r if mode else None, y)
+            if args.fp8act:
+                dps.dps_quantize_activations(x, q, scale)
+                dps.dps_linear_fp8act(enc, q, scale, p, y)
+            else:
+                dps.dps_linear(mode, enc, x, p, r if mode else None, y)
 
     stream = torch.cuda.Stream()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -72,7 +80,8 @@ def main() -> None:
     torch.cuda.synchronize()
     us = 1e3 * start.elapsed_time(stop) / args.copies
     nbytes = n * k * (2 if mode else 1) + 2 * args.M * (n + k)
-    print(f"{args.family}/{args.layer} N={n} K={k} M={args.M} {args.mode}: {us:.2f} us/launch, "
+    label = "fast+fp8act" if args.fp8act else args.mode
+    print(f"{args.family}/{args.layer} N={n} K={k} M={args.M} {label}: {us:.2f} us/launch, "
           f"{nbytes / us / 1e3:.0f} GB/s, {2 * args.M * n * k / us / 1e6:.1f} TFLOP/s, status={dps.dps_stream_status()}")
 
 
