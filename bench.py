@@ -606,6 +606,14 @@ def detail_rows(dps, workloads, torch, dev, peaks):
                           "ms_first_step_after_switch": statistics.median(after) if after else None}
         step_rows[f"M{M}"] = row
         del xs, ys, graphs
+    # the same kind of schedule derived from the memory manager model under a synthetic KV-demand trace
+    from paper_2609_34380_b200 import sum_manager
+    sm_modes, _ = sum_manager.mode_schedule_from_trace(sum_manager.kv_demand_trace(2000, 80 * 16, 5556), 80, 16, 40)
+    out["sum_manager_schedule"] = {"steps": len(sm_modes), "fast_share": sm_modes.count(0) / len(sm_modes),
+                                   "switches": sum(1 for i in range(1, len(sm_modes)) if sm_modes[i] != sm_modes[i - 1]),
+                                   "units": 80, "residual_units": 40, "blocks_per_unit": 16,
+                                   "what": "host-side model of the paper's KV block allocation algorithm driven by a seeded bursty "
+                                           "KV occupancy trace; not used for the timings above"}
     out["decoder_step_32_layers"] = {"schedule": {"steps": len(schedule), "fast_share": schedule.count(0) / len(schedule),
                                                   "switches": sum(1 for i in range(1, len(schedule)) if schedule[i] != schedule[i - 1])},
                                      "per_M": step_rows}
