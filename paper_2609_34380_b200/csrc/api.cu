@@ -165,14 +165,11 @@ dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w
     const uint8_t* r = (mode == DPS_MODE_FULL) ? w_resid : nullptr;  // fast mode never sees the pointer
     // A handful of tokens makes the layer a pure weight stream: up to 8 tokens (one MMA column group)
     // the register-streaming kernel serves it.  For 9-16 tokens the choice was measured on Llama-7B
-    // and hidden-8192 shapes: the tensor-core kernel's set-up and cluster reduction cost about 5 us
-    // per launch, its TMA stream is faster once running.  Fast mode (half the bytes, twice the
-    // MMA work per byte for the streaming kernel): streaming kernel below 2^25 weights only.
-    // Full mode: streaming kernel below 2^26 weights or with short rows (K <= 4096, few K blocks
-    // to amortise the set-up over).  Beyond 16 tokens the tcgen05 tiles take over.
-    // (The CUDA-core GEMV is kept as a cross-check.)
-    const bool stream_mid = mode == DPS_MODE_FULL ? (N * K < ((int64_t)1 << 26) || K <= 4096)
-                                                  : N * K < ((int64_t)1 << 25);
+    // and hidden-8192 shapes, in both modes: the tensor-core kernel's set-up and cluster reduction
+    // cost a few microseconds per launch, its TMA stream is faster once running; it wins from 2^25
+    // weights on (by 0-20 %), the streaming kernel below (4096 x 4096: by 15-30 %).  Beyond 16
+    // tokens the tcgen05 tiles take over.  (The CUDA-core GEMV is kept as a cross-check.)
+    const bool stream_mid = N * K < ((int64_t)1 << 25);
     const int path = forced_path();
     cudaError_t err;
     if (path == 1) err = launch_gemv(mode, enc, x, w_persist, r, y, M, N, K, stream);

@@ -274,20 +274,20 @@ cudaError_t launch_one(const __half* x, const uint8_t* p, const uint8_t* r, __ha
 template <int ENC, bool FULL>
 cudaError_t launch_enc(const __half* x, const uint8_t* p, const uint8_t* r, __half* y, int M, int64_t N, int64_t K,
                        cudaStream_t stream) {
-    // Rounds in flight per lane: 128 bytes either way (fast mode reads one plane per round).
+    // Rounds in flight per lane: 256 bytes (fast mode: 8 rounds of one plane; full mode: 4 rounds of
+    // two), two CTAs per SM.  Half as much with three CTAs per SM in full mode was the default until the
+    // first batch of weight loads moved in front of the dependency wait; since then the deeper
+    // batches measure 2-26 % faster on every Llama-7B and hidden-8192 shape but one (QKV, full mode,
+    // 8 tokens: -3 %).  DPS_STREAM_U2=0 selects the shallower batches (tuning knob).
     // Half-height blocks were measured slower for every Llama-7B shape (the kernel is bound by
     // instruction issue, and they double the MMA and activation-load instructions per weight), so
     // they stay off.
-    // Matrices with few rows (at most one wave of CTAs at three per SM) run with twice the rounds
-    // in flight per lane and two CTAs per SM: measured 10-15 % faster for N = 4096, slower for
-    // the wide layers in full mode.  DPS_STREAM_U2=0|1 overrides (tuning knob).
     static const int u_forced = [] {
         const char* e = getenv("DPS_STREAM_U2");
         return e ? atoi(e) : -1;
     }();
     constexpr int U = FULL ? 2 : 4;
-    const bool wide_batches = u_forced >= 0 ? u_forced != 0
-                                            : (N + kRowsPerBlock - 1) / kRowsPerBlock <= (int64_t)sm_count() * 3;
+    const bool wide_batches = u_forced >= 0 ? u_forced != 0 : true;
     if (wide_batches) {
         if (M <= 8) return launch_one<ENC, FULL, 1, 2 * U, false>(x, p, r, y, M, N, K, stream);
         if (M <= 16) return launch_one<ENC, FULL, 2, 2 * U, false>(x, p, r, y, M, N, K, stream);
