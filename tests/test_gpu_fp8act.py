@@ -17,7 +17,7 @@ def test_quantisation_is_bit_exact(M, K):
     x = workloads.activations(M, K, 21 + M, device=DEV)
     if M > 2:
         x[2] = 0                                   # an all-zero token
-        x[1] *= 1e-3                               # a token of small values (subnormal E4M3 codes after scaling? no: scaling is per token)
+        x[1] *= 1e-3                               # a token of small values: the scale is per token, the codes stay spread
     q, scale = dps.dps_quantize_activations(x)
     q_ref, s_ref = oracle.quantize_activations(to_np_words(x))
     assert np.array_equal(scale.cpu().numpy(), s_ref)
@@ -63,7 +63,8 @@ def test_llama_o_proj_512_tokens_and_distance_to_fp16_activations():
 
 
 def test_one_hot_activations_pick_out_fast_mode_weights():
-    """x[m] = 448-scaled one-hot: q = code of 448 at one k, scale = 1/448... -> y[m][n] = W_fast[n][k] up to FP16 rounding."""
+    """One-hot tokens: the single 1.0 quantises to the code of 448 with scale 1/448, so y[m][n] is W_fast[n][k]
+    up to one binary32 rounding of the scale and the FP16 rounding of the store."""
     N, K, M = 256, 256, 16
     w = workloads.weights(N, K, 41, device=DEV)
     for enc_req in (dps.DPS_ENC_AUTO, dps.DPS_ENC_E5M2):
