@@ -86,13 +86,12 @@ quantize_activations_kernel(const uint4* __restrict__ x, uint2* __restrict__ q, 
 }
 
 // ---- FP8 x FP8 linear ---------------------------------------------------------------------------
-constexpr int kRows = 128;      // weight rows per CTA (UMMA M)
-constexpr int kTokens = 256;    // tokens per CTA (UMMA N)
+constexpr int kRows = 128;      // weight rows per tile (UMMA M)
 constexpr int kBlockBytes = 128;                                  // K per stage (one swizzle atom of bytes)
-constexpr int kStageBytes = (kRows + kTokens) * kBlockBytes;      // 48 KB
-constexpr int kStages = 4;
 constexpr int kThreads = 192;
-constexpr uint32_t kTmemCols = 512;   // two accumulators of 256 token columns
+// Tokens per tile (UMMA N): 256, or 128 when 256-token tiles would leave SMs without one.
+__host__ __device__ constexpr int stage_bytes_fp8(int tokens) { return (kRows + tokens) * kBlockBytes; }   // 48 / 32 KB
+__host__ __device__ constexpr int stages_fp8(int tokens) { return tokens == 256 ? 4 : 6; }
 
 // Instruction descriptor for kind::f8f6f4: FP32 accumulator, K-major operands; formats 0 = E4M3, 1 = E5M2.
 __host__ __device__ constexpr uint32_t idesc_f8(int m, int n, int a_format, int b_format) {
@@ -127,9 +126,13 @@ constexpr int kEpiBytes = kEpiCols * kRows * 2;                   // 8 KB buffer
 // four epilogue warps drain the previous one -- at FP8 rates the epilogue of a 128 x 256 tile is a
 // fifth of the tile's MMA time.  The epilogue goes through a small buffer, 32 token columns at a
 // time: the stage ring never idles.
+template <int kTokens>
 __global__ void __launch_bounds__(kThreads, 1)
 fp8act_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_x,
                      const Fp8Params prm) {
+    constexpr int kStageBytes = stage_bytes_fp8(kTokens);
+    constexpr int kStages = stages_fp8(kTokens);
+    constexpr uint32_t kTmemCols = 2 * kTokens;   // two accumulators
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[kStages];
     __shared__ __align__(8) uint64_t bar_empty[kStages];
@@ -328,12 +331,15 @@ cudaError_t launch_quantize_activations(const void* x, uint8_t* q, float* scale,
     return e;
 }
 
-cudaError_t launch_linear_fp8act(int enc, const uint8_t* q, const float* scale, const uint8_t* p, void* y, int64_t M,
-                                 int64_t N, int64_t K, int* status, cudaStream_t stream) {
+namespace {
+template <int kTokens>
+cudaError_t launch_fp8_tokens(int enc, const uint8_t* q, const float* scale, const uint8_t* p, void* y, int64_t M, int64_t N,
+                              int64_t K, int* status, cudaStream_t stream) {
     static bool configured = false;
-    const size_t smem = (size_t)kStages * kStageBytes + kEpiBytes + 1024;
+    const size_t smem = (size_t)stages_fp8(kTokens) * stage_bytes_fp8(kTokens) + kEpiBytes + 1024;
+    auto kernel = fp8act_linear_kernel<kTokens>;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(fp8act_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -360,9 +366,18 @@ cudaError_t launch_linear_fp8act(int enc, const uint8_t* q, const float* scale, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, fp8act_linear_kernel, mp, mx, prm);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, mp, mx, prm);
     count_launch();
     return e;
+}
+}  // namespace
+
+cudaError_t launch_linear_fp8act(int enc, const uint8_t* q, const float* scale, const uint8_t* p, void* y, int64_t M,
+                                 int64_t N, int64_t K, int* status, cudaStream_t stream) {
+    // 256-token tiles unless they would leave SMs without a tile (few weight rows, few tokens)
+    const int64_t tiles256 = ((N + kRows - 1) / kRows) * ((M + 255) / 256);
+    if (tiles256 < sm_count() && M > 128) return launch_fp8_tokens<128>(enc, q, scale, p, y, M, N, K, status, stream);
+    return launch_fp8_tokens<256>(enc, q, scale, p, y, M, N, K, status, stream);
 }
 
 }  // namespace dps

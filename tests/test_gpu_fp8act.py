@@ -48,6 +48,18 @@ def test_linear_against_the_oracle(enc_req, N, K, M):
     assert dps.dps_stream_status() == dps.DPS_OK
 
 
+def test_more_tiles_than_sms_on_256_token_tiles():
+    """160 tiles of 128 x 256 on 148 persistent CTAs: both accumulators in use, a second tile for some CTAs."""
+    N, K, M = 4096, 272, 1280
+    w = workloads.weights(N, K, 33, device=DEV)
+    p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+    x = workloads.activations(M, K, 34, device=DEV)
+    q, scale = dps.dps_quantize_activations(x)
+    y = dps.dps_linear_fp8act(enc, q, scale, p)
+    ref = oracle.linear_fp8act(enc, to_np_bytes(q), scale.cpu().numpy(), to_np_bytes(p), threads=16)
+    assert_close_to_oracle(y, ref, "fp8act 160 tiles")
+
+
 def test_llama_o_proj_512_tokens_and_distance_to_fp16_activations():
     N, K = workloads.LLAMA7B["o"]
     w = workloads.weights(N, K, 2002, device=DEV)
