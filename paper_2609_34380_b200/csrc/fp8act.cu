@@ -33,7 +33,23 @@ using namespace sm100;
 // ---- activation quantisation ------------------------------------------------------------------
 constexpr int kQuantThreads = 256;
 
-// One CTA per token: maximum magnitude, scale, then the E4M3 codes.
+// One CTA per token: maximum magnitude, scale, then the E4M3 codes.  Rows of up to 8192 elements stay
+// in registers between the two passes (four 16-byte pieces per thread); longer rows are read again.
+constexpr int kQuantKeep = 4;
+
+__device__ __forceinline__ uint2 quantize8(const uint4& v, float sc) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t out[2] = {0u, 0u};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
+        const float2 d = make_float2(__fdiv_rn(f.x, sc), __fdiv_rn(f.y, sc));
+        const uint32_t pair = (uint32_t)__nv_cvt_float2_to_fp8x2(d, __NV_SATFINITE, __NV_E4M3);   // .x in the low byte
+        out[j >> 1] |= pair << ((j & 1) * 16);
+    }
+    return make_uint2(out[0], out[1]);
+}
+
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_activations_kernel(const uint4* __restrict__ x, uint2* __restrict__ q, float* __restrict__ scale, int64_t k8,
                             int* status) {
@@ -43,10 +59,11 @@ quantize_activations_kernel(const uint4* __restrict__ x, uint2* __restrict__ q, 
     grid_dependency_wait();   // the activations are the preceding kernel's output
     const int64_t m = blockIdx.x;
     const uint4* row = x + m * k8;
+    const bool keep = k8 <= (int64_t)kQuantKeep * kQuantThreads;
+    uint4 held[kQuantKeep];
     float amax = 0.f;
     bool bad = false;
-    for (int64_t i = threadIdx.x; i < k8; i += kQuantThreads) {
-        const uint4 v = row[i];
+    auto scan = [&](const uint4& v) {
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -55,6 +72,17 @@ quantize_activations_kernel(const uint4* __restrict__ x, uint2* __restrict__ q, 
             bad |= !(a <= 65504.f) || !(b <= 65504.f);   // Inf or NaN
             amax = fmaxf(amax, fmaxf(a, b));
         }
+    };
+    if (keep) {
+#pragma unroll
+        for (int u = 0; u < kQuantKeep; ++u) {
+            const int64_t i = (int64_t)u * kQuantThreads + threadIdx.x;
+            held[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (i < k8) held[u] = row[i];
+            scan(held[u]);
+        }
+    } else {
+        for (int64_t i = threadIdx.x; i < k8; i += kQuantThreads) scan(row[i]);
     }
     for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
     if (__syncthreads_or(bad) && threadIdx.x == 0) atomicExch(status, (int)DPS_ERR_DATA);
@@ -70,18 +98,14 @@ quantize_activations_kernel(const uint4* __restrict__ x, uint2* __restrict__ q, 
     __syncthreads();
     const float sc = s_scale;
     uint2* qrow = q + m * k8;
-    for (int64_t i = threadIdx.x; i < k8; i += kQuantThreads) {
-        const uint4 v = row[i];
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t out[2] = {0u, 0u};
+    if (keep) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
-            const float2 d = make_float2(__fdiv_rn(f.x, sc), __fdiv_rn(f.y, sc));
-            const uint32_t pair = (uint32_t)__nv_cvt_float2_to_fp8x2(d, __NV_SATFINITE, __NV_E4M3);   // .x in the low byte
-            out[j >> 1] |= pair << ((j & 1) * 16);
+        for (int u = 0; u < kQuantKeep; ++u) {
+            const int64_t i = (int64_t)u * kQuantThreads + threadIdx.x;
+            if (i < k8) qrow[i] = quantize8(held[u], sc);
         }
-        qrow[i] = make_uint2(out[0], out[1]);
+    } else {
+        for (int64_t i = threadIdx.x; i < k8; i += kQuantThreads) qrow[i] = quantize8(row[i], sc);
     }
 }
 

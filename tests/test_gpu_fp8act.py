@@ -12,8 +12,9 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-@pytest.mark.parametrize("M,K", [(1, 16), (7, 528), (300, 1040), (64, 4096)])
+@pytest.mark.parametrize("M,K", [(1, 16), (7, 528), (300, 1040), (64, 4096), (5, 8192), (3, 8208), (4, 11008)])
 def test_quantisation_is_bit_exact(M, K):
+    """Rows of up to 8192 elements are held in registers between the two passes; longer ones are read twice."""
     x = workloads.activations(M, K, 21 + M, device=DEV)
     if M > 2:
         x[2] = 0                                   # an all-zero token
