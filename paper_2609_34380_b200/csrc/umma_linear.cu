@@ -58,7 +58,7 @@ constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
 #define DPS_RB2_FAST_BK 128
 #endif
 __host__ __device__ constexpr int block_k(bool full, int tn, int rb = 1) {
-    if (rb == 2) return full ? 64 : DPS_RB2_FAST_BK;
+    if (rb == 2) return (full || tn > 128) ? 64 : DPS_RB2_FAST_BK;   // two accumulators of tn columns + four A slots in 512
     return (tn >= DPS_BK64_FROM || (full && tn <= 64)) ? 64 : 128;
 }
 // Widest tile whose split-K partial sums are pushed into a mailbox of their own; wider tiles keep
@@ -1558,6 +1558,24 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
     // DPS_DENSE_RB=1|2 overrides (tuning knob).
     const int64_t tiles_rb2 = ((N + 2 * kTileRows - 1) / (2 * kTileRows)) * ((M + 127) / 128);
     const bool rb2 = rb_forced ? rb_forced == 2 : (!FULL && tiles_rb2 > (int64_t)sm_count());
+    // ... and 192 tokens wide once there are at least two rounds of such tiles: 40 KB of planes and
+    // activations per 256 x 192 x 64 block instead of 64 KB per 256 x 128 x 128, i.e. a sixth less out of L2 per
+    // FLOP, which is what bounds the main loop (measured +5 % at 2048 tokens on the two wide Llama-7B layers,
+    // +5-8 % at 8192 on all four; with fewer tiles the coarser last round costs more than that).  Two
+    // accumulators of 192 columns and four A slots of 32 fill the tensor memory, hence 64-element K blocks.
+    // DPS_RB2_TN=128|192 overrides (tuning knob).
+    static const int rb2_tn = [] {
+        const char* e = getenv("DPS_RB2_TN");
+        return e ? atoi(e) : 0;
+    }();
+    if constexpr (!FULL) {
+        const int64_t tiles192 = ((N + 2 * kTileRows - 1) / (2 * kTileRows)) * ((M + 191) / 192);
+        // padded token columns are multiplied like real ones: at most 4 % more of them than with 128-token tiles
+        const int64_t padded192 = ((M + 191) / 192) * 192, padded128 = ((M + 127) / 128) * 128;
+        const bool wide192 = rb2_tn ? rb2_tn == 192
+                                    : tiles192 >= 2 * (int64_t)sm_count() && 25 * padded192 <= 26 * padded128;
+        if (rb2 && M > 128 && wide192) return launch_tn_rb2<ENC, FULL, 192>(x, p, r, y, M, N, K, status, stream);
+    }
     if (rb2 && M > 64) return launch_tn_rb2<ENC, FULL, 128>(x, p, r, y, M, N, K, status, stream);
     // ... unless 256-token tiles would leave half the SMs without one (few weight rows, few tokens):
     // then 128-token tiles, two CTAs per SM, win by 10-40 % (measured at 256 tokens, N = 4096 / 8192).

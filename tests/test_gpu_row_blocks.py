@@ -25,7 +25,7 @@ def _cases():
     dev = "cuda:0"
     # dense: N not a multiple of 256 (second row block ragged or absent), K with a ragged last block,
     # token counts that leave a partial last token tile
-    for (N, K, M) in [(640, 1088, 200), (128, 512, 65), (904, 2064, 300)]:
+    for (N, K, M) in [(640, 1088, 200), (128, 512, 65), (904, 2064, 300), (392, 272, 577)]:
         for forced_enc in (dps.DPS_ENC_AUTO, dps.DPS_ENC_E5M2):
             w = workloads.weights(N, K, 11 + N, device=dev)
             p, r, enc = dps.dps_split_weights(w, forced_enc)
@@ -68,7 +68,19 @@ def test_forced_two_row_blocks_in_child_process(persist):
                          text=True, timeout=600)
     assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-4000:]
     assert "all row-block cases passed" in out.stdout
-    assert out.stdout.count("ok dense") == 12 and out.stdout.count("ok grouped") == 4
+    assert out.stdout.count("ok dense") == 16 and out.stdout.count("ok grouped") == 4
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("persist", ["0", "2"])
+def test_forced_192_token_two_row_block_tiles_in_child_process(persist):
+    """Fast mode, 256 rows x 192 tokens per CTA (the launcher picks it from two rounds of such tiles on): here
+    forced on shapes with a ragged second row block, a ragged last K block and a short last token tile."""
+    env = dict(os.environ, DPS_DENSE_RB="2", DPS_RB2_TN="192", DPS_PERSIST=persist, PYTHONPATH=REPO)
+    out = subprocess.run([sys.executable, os.path.abspath(__file__)], cwd=REPO, env=env, capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-4000:]
+    assert "all row-block cases passed" in out.stdout
 
 
 @pytest.mark.gpu
