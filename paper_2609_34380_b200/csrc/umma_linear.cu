@@ -1216,6 +1216,21 @@ int persist_mode() {
     }();
     return v;
 }
+// Dense launches of SM-owning tiles with at most half as many tiles as SMs: two CTAs per tile, each
+// with one half of K, summed through the pair's shared memory (the persistent kernel's last-round
+// path, with every tile in the "last round").  Chosen when the pairs fill at least three quarters of the SMs:
+// measured +24-41 % on the Llama-7B O and down projections at 512 tokens and +18-30 % on the
+// hidden-8192 ones at 256 (64 tiles -> 128 CTAs), against 128-token tiles with a cluster split or
+// one CTA per 256-token tile; with 32 tiles (64 CTAs) it loses up to 15 %.
+// DPS_PAIR_ALL=0 never, 2 whenever the tiles allow it (tuning knob).
+bool pair_all_tiles(int64_t tiles) {
+    static const int mode = [] {
+        const char* e = getenv("DPS_PAIR_ALL");
+        return e ? atoi(e) : 1;
+    }();
+    if (mode == 0 || tiles < 1 || 2 * tiles > sm_count()) return false;
+    return mode == 2 || 8 * tiles >= 3 * (int64_t)sm_count();
+}
 bool use_persistent(int64_t tiles) { return persist_mode() == 2 || (persist_mode() == 1 && tiles > sm_count()); }
 
 // Persistent launch: one CTA per SM (or fewer, if there are fewer tiles) walks `tiles` tiles.
@@ -1248,6 +1263,7 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
     prm.x_offset = 0;
     prm.pair_min = pair_min_depth();
     int64_t grid = tiles < sm_count() ? tiles : sm_count();
+
     // CTA pairs (clusters of two) so that the tiles of a short last round can be shared out as halves
     // of K, summed through the pair's shared memory; the FP32 partial tile must fit over the ring.
     // DPS_TAIL_KSPLIT=0 launches single CTAs (tuning knob).
@@ -1256,6 +1272,11 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
         return e ? atoi(e) : 1;
     }();
     const bool ksplit_enabled = ksplit_mode != 0;
+    // Dense launches with at most half as many tiles as SMs: two CTAs per tile, each with one half of K
+    // (the kernel treats all of them as the "last round").
+    if (!GROUPED && ksplit_mode == 1 && pair_all_tiles(tiles) &&
+        (size_t)TN * kTileRows * RB * 4 <= (size_t)stages * kStage)
+        grid = 2 * tiles;
     const bool pairs = ksplit_enabled && grid >= 2 && (size_t)TN * kTileRows * RB * 4 <= (size_t)stages * kStage;
     if (pairs) grid &= ~(int64_t)1;
     prm.split = (pairs && ksplit_mode == 1) ? 2 : 1;
@@ -1425,7 +1446,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     prm.status = status;
     if constexpr (kCtasPerSm == 1) {
         // a tile shape that owns its SM: with more tiles than SMs, let one CTA per SM walk them
-        if (split == 1 && use_persistent(row_tiles * tok_tiles))
+        if ((split == 1 && use_persistent(row_tiles * tok_tiles)) || pair_all_tiles(row_tiles * tok_tiles))
             return launch_persistent<ENC, FULL, TN, false, 1>(mp, mr, mx, prm, GroupedParams{}, row_tiles * tok_tiles,
                                                              x, M, stream);
     }
@@ -1580,6 +1601,9 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
     // ... unless 256-token tiles would leave half the SMs without one (few weight rows, few tokens):
     // then 128-token tiles, two CTAs per SM, win by 10-40 % (measured at 256 tokens, N = 4096 / 8192).
     const int64_t tiles256 = ((N + kTileRows - 1) / kTileRows) * ((M + 255) / 256);
+    // few 256-token tiles, but enough for CTA pairs (halves of K) to fill most SMs
+    if (!tn_forced && M > 128 && pair_all_tiles(tiles256))
+        return launch_tn<ENC, FULL, 256>(x, p, r, y, M, N, K, status, stream);
     const bool wide = tn_forced ? tn_forced == 256
                                 : (FULL ? M > 128 : (M > 128 && M <= 256)) && 2 * tiles256 > (int64_t)sm_count();
     if (!wide) return launch_tn<ENC, FULL, 128>(x, p, r, y, M, N, K, status, stream);

@@ -84,6 +84,16 @@ def test_forced_192_token_two_row_block_tiles_in_child_process(persist):
 
 
 @pytest.mark.gpu
+def test_forced_k_halves_for_every_tile_in_child_process():
+    """Few 256-token tiles: two CTAs per tile, each with one half of K (forced; 1 to 8 tiles here)."""
+    env = dict(os.environ, DPS_PAIR_ALL="2", DPS_FORCE_TN="256", PYTHONPATH=REPO)
+    out = subprocess.run([sys.executable, os.path.abspath(__file__)], cwd=REPO, env=env, capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-4000:]
+    assert "all row-block cases passed" in out.stdout
+
+
+@pytest.mark.gpu
 def test_forced_persistent_kernel_with_default_tiles_in_child_process():
     """256-token tiles (forced: the shapes here are small) walked by the persistent kernel."""
     env = dict(os.environ, DPS_PERSIST="2", DPS_FORCE_TN="256", PYTHONPATH=REPO)
