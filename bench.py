@@ -494,6 +494,29 @@ def detail_rows(dps, workloads, torch, dev, peaks):
     del planes
     torch.cuda.empty_cache()
 
+    # ---- rounded nests (extension): full mode pays one saturating subtract per weight pair ----
+    rn = {}
+    n, k = workloads.LLAMA7B["qkv"]
+    wts = [workloads.weights(n, k, 2001 + 100 * c, device=dev) for c in range(4)]
+    for label, enc_req in (("truncated", dps.DPS_ENC_E4M3), ("rounded", dps.DPS_ENC_E4M3_RN)):
+        pl = [dps.dps_split_weights(w, enc_req) for w in wts]
+        for M in (8, 2048):
+            x = workloads.activations(M, k, 3001, device=dev)
+            y = torch.empty((M, n), dtype=torch.float16, device=dev)
+            ms, _ = _time_graph(torch, stream, lambda: [dps.dps_linear(dps.DPS_MODE_FULL, e, x, p, r, y) for p, r, e in pl],
+                                iters=5, warm=2)
+            if M == 8:
+                rn[f"qkv_M8_full_{label}_GB/s"] = 4 * linear_bytes(True, M, n, k) / (ms * 1e-3) / 1e9
+            else:
+                rn[f"qkv_M2048_full_{label}_TFLOP/s"] = 4 * 2 * M * n * k / (ms * 1e-3) / 1e12
+            del x, y
+        del pl
+    rn["what"] = ("Llama-7B QKV, 4 weight copies in rotation, full mode, E4M3 nest against its rounded variant "
+                  "(fast mode runs the same kernels on either plane)")
+    out["rounded_nest"] = rn
+    del wts
+    torch.cuda.empty_cache()
+
     # ---- MoE (config 4) ----
     moe = {}
     E, T = workloads.MIXTRAL_EXPERTS, workloads.MIXTRAL_TOKENS

@@ -71,7 +71,13 @@ typedef enum {
 } dps_status;
 
 typedef enum { DPS_MODE_FAST = 0, DPS_MODE_FULL = 1 } dps_mode;
-typedef enum { DPS_ENC_AUTO = 0, DPS_ENC_E4M3 = 1, DPS_ENC_E5M2 = 2 } dps_encoding;
+typedef enum {
+    DPS_ENC_AUTO = 0,
+    DPS_ENC_E4M3 = 1,
+    DPS_ENC_E5M2 = 2,
+    DPS_ENC_E4M3_RN = 3, /* rounded nests, see below */
+    DPS_ENC_E5M2_RN = 4
+} dps_encoding;
 
 /*
  * Nested split (paper: "Persistent Region" paragraph).  With b the FP16 word
@@ -80,8 +86,18 @@ typedef enum { DPS_ENC_AUTO = 0, DPS_ENC_E4M3 = 1, DPS_ENC_E5M2 = 2 } dps_encodi
  *   E4M3: P = s e[3:0] m[9:7]          R = 0 m[6:0]      (needs b[14] == 0 everywhere)
  * Bits are selected, never rounded, so (P, R) rebuilds W exactly.
  *
+ * Rounded nests (an extension: the paper describes the bit selection only).  DPS_ENC_E5M2_RN and
+ * DPS_ENC_E4M3_RN store the same fields of b' = b + 0x0080 (E5M2) or b + 0x0040 (E4M3), i.e. of
+ * the word plus half a unit of the last bit P keeps.  P is then the FP8 value NEAREST to the
+ * weight (ties away from zero) instead of the next one towards zero, which removes the
+ * shrinking bias of fast mode, and join(P, R) - the same constant still rebuilds W exactly.
+ * Legal iff no b' reaches an Inf / NaN code: max|b & 0x7FFF| + 0x80 < 0x7C00 (E5M2_RN),
+ * + 0x40 < 0x3F80 (E4M3_RN).  Never chosen by AUTO.  Accepted by dps_split_weights,
+ * dps_reconstruct, dps_linear and dps_linear_fp8act; the grouped calls take the two
+ * truncated encodings only.
+ *
  * w_fp16: device, rows*cols FP16 words.  w_persist, w_resid: device, rows*cols bytes each.
- * enc_inout: HOST int32.  On entry DPS_ENC_AUTO, DPS_ENC_E4M3 or DPS_ENC_E5M2; on return
+ * enc_inout: HOST int32.  On entry DPS_ENC_AUTO or one of the four encodings; on return
  * the encoding that was used.
  *   AUTO  -> E4M3 iff every word has b[14] == 0 and max|w| <= 1.75, else E5M2.  The
  *            statistics pass needs its result on the host, so this variant SYNCHRONISES
@@ -90,6 +106,7 @@ typedef enum { DPS_ENC_AUTO = 0, DPS_ENC_E4M3 = 1, DPS_ENC_E5M2 = 2 } dps_encodi
  *            or would produce the byte 0x7F/0xFF the call returns DPS_ERR_DATA with both
  *            planes untouched.
  *   E5M2  -> always legal, never synchronises.
+ *   E4M3_RN, E5M2_RN -> checked like E4M3 (synchronise; DPS_ERR_DATA if not legal).
  * rows*cols == 0 returns DPS_OK (AUTO then reports E4M3).  cols must be a multiple of 16.
  */
 DPS_API dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_resid,
@@ -99,7 +116,8 @@ DPS_API dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uin
  * Reconstruction (paper: "Overall concept" paragraph, full mode): the inverse of the
  * split, W = join(P, R), bit-exact.  Bit 7 of an E4M3 residual byte is ignored.
  * w_resid == NULL rebuilds the fast-mode weights instead (residual taken as zero).
- * enc must be DPS_ENC_E4M3 or DPS_ENC_E5M2.  Never synchronises.
+ * (for a rounded nest: the values of its persistent bytes, i.e. the rounded weights).
+ * enc must be one of the four encodings, never AUTO.  Never synchronises.
  */
 DPS_API dps_status dps_reconstruct(const uint8_t* w_persist, const uint8_t* w_resid, void* w_fp16_out,
                            int64_t rows, int64_t cols, int32_t enc, void* cuda_stream);
@@ -109,7 +127,7 @@ DPS_API dps_status dps_reconstruct(const uint8_t* w_persist, const uint8_t* w_re
  *   y[M][N] (FP16) = x[M][K] (FP16) * W_eff^T, FP32 accumulation, one FP16 rounding at the
  *   store.  FULL: W_eff = join(P, R), the original FP16 weights.  FAST: W_eff = join(P, 0);
  *   w_resid is never dereferenced and may be NULL or point at unrelated data.
- * enc must be E4M3 or E5M2 (the value dps_split_weights reported).  M == 0 returns DPS_OK
+ * enc must be one of the four encodings (the value dps_split_weights reported).  M == 0 returns DPS_OK
  * without a launch.  Never synchronises, never allocates.  Results are deterministic: the
  * same inputs give the same bits on every call.
  */

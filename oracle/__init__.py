@@ -23,6 +23,7 @@ import numpy as np
 
 MODE_FAST, MODE_FULL = 0, 1
 ENC_AUTO, ENC_E4M3, ENC_E5M2 = 0, 1, 2
+ENC_E4M3_RN, ENC_E5M2_RN = 3, 4          # rounded nests (an extension, see dps_oracle.c)
 OK, ERR_ARG, ERR_DATA = 0, 1, 8
 
 _HERE = Path(__file__).resolve().parent
@@ -57,6 +58,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_select_encoding.argtypes = [vp, i64]
         L.oracle_e4m3_legal.restype = ctypes.c_int
         L.oracle_e4m3_legal.argtypes = [vp, i64]
+        L.oracle_rounded_legal.restype = ctypes.c_int
+        L.oracle_rounded_legal.argtypes = [vp, i64, ctypes.c_int]
         L.oracle_split.restype = ctypes.c_int
         L.oracle_split.argtypes = [vp, vp, vp, i64, ctypes.c_int]
         L.oracle_reconstruct.restype = ctypes.c_int
@@ -128,6 +131,12 @@ def select_encoding(w) -> int:
 def e4m3_legal(w) -> bool:
     w = _words(w)
     return bool(lib().oracle_e4m3_legal(_ptr(w), w.size))
+
+
+def rounded_legal(w, enc: int) -> bool:
+    """Whether a rounded nest (ENC_E4M3_RN / ENC_E5M2_RN) may encode these weights."""
+    w = _words(w)
+    return bool(lib().oracle_rounded_legal(_ptr(w), w.size, enc))
 
 
 def split(w, enc: int):

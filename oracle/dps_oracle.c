@@ -40,7 +40,7 @@
 #include <string.h>
 
 enum { ORACLE_MODE_FAST = 0, ORACLE_MODE_FULL = 1 };
-enum { ORACLE_ENC_AUTO = 0, ORACLE_ENC_E4M3 = 1, ORACLE_ENC_E5M2 = 2 };
+enum { ORACLE_ENC_AUTO = 0, ORACLE_ENC_E4M3 = 1, ORACLE_ENC_E5M2 = 2, ORACLE_ENC_E4M3_RN = 3, ORACLE_ENC_E5M2_RN = 4 };
 enum { ORACLE_OK = 0, ORACLE_ERR_ARG = 1, ORACLE_ERR_DATA = 8 };
 
 /* ---- IEEE-754 binary16 <-> binary64, written from the format definition ---- */
@@ -111,9 +111,43 @@ int oracle_e4m3_legal(const uint16_t* w, int64_t n) {
     return 1;
 }
 
+/* ---- rounded nests (an extension; the paper describes bit selection only) ----
+ * The stored pair is the truncated split of b' = b + h, h = half a unit of the last bit the
+ * persistent byte keeps (E5M2: 0x0080, E4M3: 0x0040).  The persistent byte is then the FP8 value
+ * nearest to the weight, ties away from zero (pinned in the tests against that definition), and
+ * join(P, R) - h gives b back.  Legal iff no b' reaches an Inf / NaN code. */
+static int is_rounded(int enc) { return enc == ORACLE_ENC_E4M3_RN || enc == ORACLE_ENC_E5M2_RN; }
+static int base_of(int enc) {
+    return enc == ORACLE_ENC_E4M3_RN ? ORACLE_ENC_E4M3 : enc == ORACLE_ENC_E5M2_RN ? ORACLE_ENC_E5M2 : enc;
+}
+static unsigned half_unit(int enc) { return enc == ORACLE_ENC_E4M3_RN ? 0x40u : enc == ORACLE_ENC_E5M2_RN ? 0x80u : 0u; }
+static int known_enc(int enc) { return enc >= ORACLE_ENC_E4M3 && enc <= ORACLE_ENC_E5M2_RN; }
+
+int oracle_rounded_legal(const uint16_t* w, int64_t n, int enc) {
+    if (!is_rounded(enc)) return 0;
+    const unsigned limit = enc == ORACLE_ENC_E5M2_RN ? 0x7C00u : 0x3F80u;
+    for (int64_t i = 0; i < n; ++i)
+        if ((w[i] & 0x7FFFu) + half_unit(enc) >= limit) return 0;
+    return 1;
+}
+
 /* ---- split / reconstruct / fast value: one element ---- */
 
+static void split_trunc(uint16_t b, int enc, uint8_t* p, uint8_t* r);
+static uint16_t join_trunc(uint8_t p, uint8_t r, int enc);
+
 static void split_one(uint16_t b, int enc, uint8_t* p, uint8_t* r) {
+    split_trunc((uint16_t)(b + half_unit(enc)), base_of(enc), p, r);
+}
+
+/* residual == NULL-like use: the callers pass r = 0 AND full = 0 for the fast-mode value, which is
+ * the value of the persistent byte itself, also for a rounded nest. */
+static uint16_t join_one_mode(uint8_t p, uint8_t r, int enc, int full) {
+    if (!full) return join_trunc(p, 0, base_of(enc));
+    return (uint16_t)(join_trunc(p, r, base_of(enc)) - half_unit(enc));
+}
+
+static void split_trunc(uint16_t b, int enc, uint8_t* p, uint8_t* r) {
     unsigned s = (b >> 15) & 1u, e = (b >> 10) & 0x1Fu, m = b & 0x3FFu;
     if (enc == ORACLE_ENC_E5M2) {
         *p = (uint8_t)((s << 7) | (e << 2) | (m >> 8));   /* s e4..e0 m9 m8 */
@@ -124,7 +158,7 @@ static void split_one(uint16_t b, int enc, uint8_t* p, uint8_t* r) {
     }
 }
 
-static uint16_t join_one(uint8_t p, uint8_t r, int enc) {
+static uint16_t join_trunc(uint8_t p, uint8_t r, int enc) {
     unsigned s = (p >> 7) & 1u;
     if (enc == ORACLE_ENC_E5M2) {
         unsigned e = (p >> 2) & 0x1Fu, mh = p & 3u;
@@ -138,23 +172,24 @@ static uint16_t join_one(uint8_t p, uint8_t r, int enc) {
 /* FP16 -> (P, R).  enc must be E4M3 or E5M2 (the caller resolves AUTO with
  * oracle_select_encoding).  An illegal E4M3 request leaves the planes alone. */
 int oracle_split(const uint16_t* w, uint8_t* p, uint8_t* r, int64_t n, int enc) {
-    if (enc != ORACLE_ENC_E4M3 && enc != ORACLE_ENC_E5M2) return ORACLE_ERR_ARG;
+    if (!known_enc(enc)) return ORACLE_ERR_ARG;
     if (enc == ORACLE_ENC_E4M3 && !oracle_e4m3_legal(w, n)) return ORACLE_ERR_DATA;
+    if (is_rounded(enc) && !oracle_rounded_legal(w, n, enc)) return ORACLE_ERR_DATA;
     for (int64_t i = 0; i < n; ++i) split_one(w[i], enc, &p[i], &r[i]);
     return ORACLE_OK;
 }
 
 /* (P, R) -> original FP16 words (full mode's weights). */
 int oracle_reconstruct(const uint8_t* p, const uint8_t* r, uint16_t* w, int64_t n, int enc) {
-    if (enc != ORACLE_ENC_E4M3 && enc != ORACLE_ENC_E5M2) return ORACLE_ERR_ARG;
-    for (int64_t i = 0; i < n; ++i) w[i] = join_one(p[i], r[i], enc);
+    if (!known_enc(enc)) return ORACLE_ERR_ARG;
+    for (int64_t i = 0; i < n; ++i) w[i] = join_one_mode(p[i], r[i], enc, 1);
     return ORACLE_OK;
 }
 
 /* P alone -> FP16 words of the fast-mode weights (residual taken as zero). */
 int oracle_fast_words(const uint8_t* p, uint16_t* w, int64_t n, int enc) {
-    if (enc != ORACLE_ENC_E4M3 && enc != ORACLE_ENC_E5M2) return ORACLE_ERR_ARG;
-    for (int64_t i = 0; i < n; ++i) w[i] = join_one(p[i], 0, enc);
+    if (!known_enc(enc)) return ORACLE_ERR_ARG;
+    for (int64_t i = 0; i < n; ++i) w[i] = join_one_mode(p[i], 0, enc, 0);
     return ORACLE_OK;
 }
 
@@ -162,8 +197,8 @@ int oracle_fast_words(const uint8_t* p, uint16_t* w, int64_t n, int enc) {
 
 /* Effective weight of element i of a plane pair, as a double. */
 static double eff_weight(int mode, int enc, const uint8_t* p, const uint8_t* r, int64_t i) {
-    uint8_t res = (mode == ORACLE_MODE_FULL) ? r[i] : 0; /* fast mode never reads r */
-    return oracle_half_to_double(join_one(p[i], res, enc));
+    if (mode != ORACLE_MODE_FULL) return oracle_half_to_double(join_one_mode(p[i], 0, enc, 0)); /* fast mode never reads r */
+    return oracle_half_to_double(join_one_mode(p[i], r[i], enc, 1));
 }
 
 /* y_ref[m][n] = sum_k x[m][k] * W_eff[n][k], FP64, k ascending.
@@ -174,7 +209,7 @@ static double eff_weight(int mode, int enc, const uint8_t* p, const uint8_t* r, 
 int oracle_linear(int mode, int enc, const uint16_t* x, const uint8_t* p, const uint8_t* r,
                   double* y_ref, uint16_t* y_half, int64_t M, int64_t N, int64_t K, int threads) {
     if (mode != ORACLE_MODE_FAST && mode != ORACLE_MODE_FULL) return ORACLE_ERR_ARG;
-    if (enc != ORACLE_ENC_E4M3 && enc != ORACLE_ENC_E5M2) return ORACLE_ERR_ARG;
+    if (!known_enc(enc)) return ORACLE_ERR_ARG;
     if (M == 0 || N == 0) return ORACLE_OK;
     double* xd = (double*)malloc(sizeof(double) * (size_t)(M * K > 0 ? M * K : 1));
     if (!xd) return ORACLE_ERR_ARG;
@@ -205,7 +240,7 @@ int oracle_linear_at(int mode, int enc, const uint16_t* x, const uint8_t* p, con
                      int64_t M, int64_t N, int64_t K, const int64_t* ms, const int64_t* ns,
                      int64_t count, double* out) {
     if (mode != ORACLE_MODE_FAST && mode != ORACLE_MODE_FULL) return ORACLE_ERR_ARG;
-    if (enc != ORACLE_ENC_E4M3 && enc != ORACLE_ENC_E5M2) return ORACLE_ERR_ARG;
+    if (!known_enc(enc)) return ORACLE_ERR_ARG;
     for (int64_t i = 0; i < count; ++i) {
         int64_t m = ms[i], n = ns[i];
         if (m < 0 || m >= M || n < 0 || n >= N) return ORACLE_ERR_ARG;
@@ -320,7 +355,7 @@ int oracle_quantize_activations(const uint16_t* x, uint8_t* q, float* scale, int
 /* y_ref[m][n] = scale[m] * sum_k value(q[m][k]) * W_fast[n][k], FP64, k ascending. */
 int oracle_linear_fp8act(int enc, const uint8_t* q, const float* scale, const uint8_t* p, double* y_ref, int64_t M,
                          int64_t N, int64_t K, int threads) {
-    if (enc != ORACLE_ENC_E4M3 && enc != ORACLE_ENC_E5M2) return ORACLE_ERR_ARG;
+    if (!known_enc(enc)) return ORACLE_ERR_ARG;
     if (M == 0 || N == 0) return ORACLE_OK;
     double* xd = (double*)malloc(sizeof(double) * (size_t)(M * K > 0 ? M * K : 1));
     if (!xd) return ORACLE_ERR_ARG;
@@ -344,4 +379,4 @@ int oracle_linear_fp8act(int enc, const uint8_t* q, const float* scale, const ui
     return ORACLE_OK;
 }
 
-int oracle_version(void) { return 2; }
+int oracle_version(void) { return 3; }

@@ -5,6 +5,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "bits.cuh"
 #include "dps_internal.h"
 
 namespace dps {
@@ -86,13 +87,19 @@ int sm_count() {
 
 using namespace dps;
 
+namespace {
+bool known_encoding(int32_t enc) {
+    return enc == DPS_ENC_E4M3 || enc == DPS_ENC_E5M2 || enc == DPS_ENC_E4M3_RN || enc == DPS_ENC_E5M2_RN;
+}
+}  // namespace
+
 extern "C" {
 
 dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_resid, int64_t rows, int64_t cols,
                              int32_t* enc_inout, void* cuda_stream) {
     if (enc_inout == nullptr) return DPS_ERR_NULL;
     const int32_t req = *enc_inout;
-    if (req != DPS_ENC_AUTO && req != DPS_ENC_E4M3 && req != DPS_ENC_E5M2) return DPS_ERR_ENCODING;
+    if (req != DPS_ENC_AUTO && !known_encoding(req)) return DPS_ERR_ENCODING;
     if (rows < 0 || cols < 0 || (cols % 16) != 0) return DPS_ERR_SHAPE;
     if (rows > 0 && cols > 0 && rows > INT64_MAX / cols) return DPS_ERR_SHAPE;
     const int64_t n = rows * cols;
@@ -112,6 +119,8 @@ dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_
         // MSB set is >= 0x4000, so one maximum answers both questions:
         //   AUTO  -> E4M3 iff max <= 0x3F00 (|w| <= 1.75), else E5M2
         //   E4M3  -> legal iff max <  0x3F80 (exponent MSB clear and the byte is not 0x7F/0xFF)
+        //   rounded nests: the same limits must hold after half a unit of the last kept bit is added
+        //     E4M3_RN -> legal iff max + 0x40 < 0x3F80;  E5M2_RN -> legal iff max + 0x80 < 0x7C00 (no Inf code)
         std::lock_guard<std::mutex> lock(g_stat_mutex);
         unsigned maxmag = 0;
         if (cudaMemsetAsync(d->stat, 0, sizeof(unsigned), stream) != cudaSuccess) return DPS_ERR_CUDA;
@@ -121,7 +130,9 @@ dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_
             return DPS_ERR_CUDA;
         if (cudaStreamSynchronize(stream) != cudaSuccess) return DPS_ERR_CUDA;
         if (req == DPS_ENC_AUTO) enc = (maxmag <= 0x3F00u) ? DPS_ENC_E4M3 : DPS_ENC_E5M2;
-        else if (maxmag >= 0x3F80u) return DPS_ERR_DATA;
+        else if (req == DPS_ENC_E4M3 && maxmag >= 0x3F80u) return DPS_ERR_DATA;
+        else if (req == DPS_ENC_E4M3_RN && maxmag + 0x40u >= 0x3F80u) return DPS_ERR_DATA;
+        else if (req == DPS_ENC_E5M2_RN && maxmag + 0x80u >= 0x7C00u) return DPS_ERR_DATA;
     }
     if (launch_split(static_cast<const uint16_t*>(w_fp16), w_persist, w_resid, n, enc, stream) != cudaSuccess)
         return DPS_ERR_CUDA;
@@ -131,7 +142,7 @@ dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_
 
 dps_status dps_reconstruct(const uint8_t* w_persist, const uint8_t* w_resid, void* w_fp16_out, int64_t rows,
                            int64_t cols, int32_t enc, void* cuda_stream) {
-    if (enc != DPS_ENC_E4M3 && enc != DPS_ENC_E5M2) return DPS_ERR_ENCODING;
+    if (!known_encoding(enc)) return DPS_ERR_ENCODING;
     if (rows < 0 || cols < 0 || (cols % 16) != 0) return DPS_ERR_SHAPE;
     if (rows > 0 && cols > 0 && rows > INT64_MAX / cols) return DPS_ERR_SHAPE;
     const int64_t n = rows * cols;
@@ -150,7 +161,7 @@ dps_status dps_reconstruct(const uint8_t* w_persist, const uint8_t* w_resid, voi
 dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w_persist, const uint8_t* w_resid,
                       void* y, int64_t M, int64_t N, int64_t K, void* cuda_stream) {
     if (mode != DPS_MODE_FAST && mode != DPS_MODE_FULL) return DPS_ERR_MODE;
-    if (enc != DPS_ENC_E4M3 && enc != DPS_ENC_E5M2) return DPS_ERR_ENCODING;
+    if (!known_encoding(enc)) return DPS_ERR_ENCODING;
     if (M < 0 || N <= 0 || K <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
     if (N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31) || M > ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
     if (M == 0) return DPS_OK;
@@ -244,7 +255,8 @@ dps_status dps_quantize_activations(const void* x, uint8_t* x_fp8, float* scale,
 
 dps_status dps_linear_fp8act(int32_t enc, const uint8_t* x_fp8, const float* scale, const uint8_t* w_persist, void* y,
                              int64_t M, int64_t N, int64_t K, void* cuda_stream) {
-    if (enc != DPS_ENC_E4M3 && enc != DPS_ENC_E5M2) return DPS_ERR_ENCODING;
+    if (!known_encoding(enc)) return DPS_ERR_ENCODING;
+    enc = base_enc(enc);   // the persistent byte of a rounded nest is an FP8 value like any other
     if (M < 0 || N <= 0 || K <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
     if (N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31) || M > ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
     if (M == 0) return DPS_OK;

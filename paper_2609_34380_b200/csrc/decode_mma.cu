@@ -304,6 +304,9 @@ cudaError_t launch_decode_mma(int mode, int enc, const void* x, const uint8_t* p
     const __half* xh = static_cast<const __half*>(x);
     __half* yh = static_cast<__half*>(y);
     const bool full = mode == DPS_MODE_FULL;
+    if (!full) enc = base_enc(enc);   // fast mode: the persistent byte of a rounded nest is an FP8 value like any other
+    if (enc == kEncE4M3R) return launch_enc<kEncE4M3R, true>(xh, p, r, yh, (int)M, N, K, stream);
+    if (enc == kEncE5M2R) return launch_enc<kEncE5M2R, true>(xh, p, r, yh, (int)M, N, K, stream);
     if (enc == kEncE4M3)
         return full ? launch_enc<kEncE4M3, true>(xh, p, r, yh, (int)M, N, K, stream)
                     : launch_enc<kEncE4M3, false>(xh, p, r, yh, (int)M, N, K, stream);

@@ -130,14 +130,13 @@ cudaError_t launch_magnitude_stat(const uint16_t* w, int64_t n, unsigned* stat, 
 cudaError_t launch_split(const uint16_t* w, uint8_t* p, uint8_t* r, int64_t n, int enc, cudaStream_t stream) {
     int64_t n8 = n / 8;
     int grid = stream_grid((n8 + kItemsPerStep - 1) / kItemsPerStep);
-    if (enc == kEncE4M3)
-        split_kernel<kEncE4M3><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint4*>(w),
-                                                               reinterpret_cast<uint2*>(p),
-                                                               reinterpret_cast<uint2*>(r), n8);
-    else
-        split_kernel<kEncE5M2><<<grid, kThreads, 0, stream>>>(reinterpret_cast<const uint4*>(w),
-                                                               reinterpret_cast<uint2*>(p),
-                                                               reinterpret_cast<uint2*>(r), n8);
+    const uint4* ww = reinterpret_cast<const uint4*>(w);
+    uint2* pp = reinterpret_cast<uint2*>(p);
+    uint2* rr = reinterpret_cast<uint2*>(r);
+    if (enc == kEncE4M3) split_kernel<kEncE4M3><<<grid, kThreads, 0, stream>>>(ww, pp, rr, n8);
+    else if (enc == kEncE5M2) split_kernel<kEncE5M2><<<grid, kThreads, 0, stream>>>(ww, pp, rr, n8);
+    else if (enc == kEncE4M3R) split_kernel<kEncE4M3R><<<grid, kThreads, 0, stream>>>(ww, pp, rr, n8);
+    else split_kernel<kEncE5M2R><<<grid, kThreads, 0, stream>>>(ww, pp, rr, n8);
     count_launch();
     plane_fence_kernel<<<1, 32, 0, stream>>>();
     count_launch();
@@ -151,12 +150,18 @@ cudaError_t launch_reconstruct(const uint8_t* p, const uint8_t* r, uint16_t* w, 
     const uint2* pp = reinterpret_cast<const uint2*>(p);
     const uint2* rr = reinterpret_cast<const uint2*>(r);
     uint4* ww = reinterpret_cast<uint4*>(w);
+    // without the residual plane the rounded nests read like their truncated siblings: P is an FP8 value
+    if (!r) enc = base_enc(enc);
     if (enc == kEncE4M3) {
         if (r) reconstruct_kernel<kEncE4M3, true><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
         else reconstruct_kernel<kEncE4M3, false><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
-    } else {
+    } else if (enc == kEncE5M2) {
         if (r) reconstruct_kernel<kEncE5M2, true><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
         else reconstruct_kernel<kEncE5M2, false><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
+    } else if (enc == kEncE4M3R) {
+        reconstruct_kernel<kEncE4M3R, true><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
+    } else {
+        reconstruct_kernel<kEncE5M2R, true><<<grid, kThreads, 0, stream>>>(pp, rr, ww, n8);
     }
     count_launch();
     return cudaGetLastError();

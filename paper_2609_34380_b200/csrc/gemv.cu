@@ -75,7 +75,10 @@ cudaError_t launch_gemv(int mode, int enc, const void* x, const uint8_t* p, cons
         const __half* xs = xh + m0 * K;
         __half* ys = yh + m0 * N;
         cudaError_t e;
-        if (enc == kEncE4M3)
+        const int enc_here = full ? enc : base_enc(enc);
+        if (enc_here == kEncE4M3R) e = launch_tokens<kEncE4M3R, true>(xs, p, r, ys, mc, N, K, stream);
+        else if (enc_here == kEncE5M2R) e = launch_tokens<kEncE5M2R, true>(xs, p, r, ys, mc, N, K, stream);
+        else if (enc_here == kEncE4M3)
             e = full ? launch_tokens<kEncE4M3, true>(xs, p, r, ys, mc, N, K, stream)
                      : launch_tokens<kEncE4M3, false>(xs, p, r, ys, mc, N, K, stream);
         else

@@ -1757,6 +1757,9 @@ cudaError_t launch_umma_grouped(int mode, const uint32_t* e5m2_mask, const void*
 cudaError_t launch_umma_linear(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
                                int64_t M, int64_t N, int64_t K, int* status, cudaStream_t stream) {
     const bool full = mode == DPS_MODE_FULL;
+    if (!full) enc = base_enc(enc);   // fast mode reads the persistent byte of a rounded nest like any other
+    if (enc == kEncE4M3R) return launch_enc<kEncE4M3R, true>(x, p, r, y, M, N, K, status, stream);
+    if (enc == kEncE5M2R) return launch_enc<kEncE5M2R, true>(x, p, r, y, M, N, K, status, stream);
     if (enc == kEncE4M3)
         return full ? launch_enc<kEncE4M3, true>(x, p, r, y, M, N, K, status, stream)
                     : launch_enc<kEncE4M3, false>(x, p, r, y, M, N, K, status, stream);
