@@ -316,6 +316,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     __shared__ __align__(8) uint64_t bar_d_full;
     __shared__ __align__(8) uint64_t bar_x_full[kMaxXSlots];
     __shared__ uint32_t tmem_base_slot;
+    __shared__ int s_rows[GROUPED ? TN : 1];   // grouped launches: row ids of the tile's tokens
 
     grid_launch_dependents();  // the next kernel's prologue may overlap this kernel's tail
     DPS_CTA_STAMP(0);
@@ -595,6 +596,9 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         // 64-byte rows: chunk index ^= (row / 2) % 4
         zc.sw = kBlockK == 128 ? (uint32_t)(row & 7) : (uint32_t)((row >> 1) & 3);
         zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
+        // grouped launches: the callers' row ids of the tile's tokens, fetched before the zip loop (which
+        // hides the latency) rather than in front of every store of the epilogue
+        if (GROUPED && (int)threadIdx.x - 64 < tile_tokens) s_rows[threadIdx.x - 64] = gp.sorted_rows[m0 + (int)threadIdx.x - 64];
         if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2)) {
             // encoding known only at run time (one per expert): uniform branch per CTA
             ZipState zst;
@@ -648,7 +652,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                     const int c = item / kChunks, q = item % kChunks;
                     const int n = n0 + q * 8;
                     if (n >= prm.N) continue;                     // N is a multiple of 8: a piece is in or out
-                    const int m = GROUPED ? gp.sorted_rows[m0 + c] : m0 + c;
+                    const int m = GROUPED ? s_rows[c] : m0 + c;
                     uint4 val;
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                                  : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
@@ -858,6 +862,8 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     __shared__ __align__(8) uint64_t bar_d_empty;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int s_rows[GROUPED ? TN : 1];   // grouped launches: row ids of the current tile's tokens
+    static_assert(!GROUPED || TN <= kZipThreads, "one zip thread per token fetches its row id");
 
     grid_launch_dependents();
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -1008,6 +1014,10 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
             const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
             if (t.tile_tokens <= 0) continue;
             zc.num_kb = khalf < 0 ? num_kb : (khalf == 0 ? num_kb / 2 : num_kb - num_kb / 2);
+            // Grouped launches: the callers' row ids of this tile's tokens, fetched now (the zip loop hides
+            // the latency) instead of one dependent global load in front of every store of the epilogue --
+            // that gather cost 10 % of a fast-mode MoE layer.  The epilogue's barriers order the accesses.
+            if (GROUPED && zt < t.tile_tokens) s_rows[zt] = gp.sorted_rows[t.m0 + zt];
             if (ok) {
                 if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2))
                     ok = t.e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
@@ -1078,7 +1088,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                         const int c = item / kChunks, qq = item % kChunks;
                         const int n = t.n0 + qq * 8;
                         if (n >= prm.N) continue;                     // N is a multiple of 8
-                        const int m = GROUPED ? gp.sorted_rows[t.m0 + c0 + c] : t.m0 + c0 + c;
+                        const int m = GROUPED ? s_rows[c0 + c] : t.m0 + c0 + c;
                         uint4 val;
                         asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                                      : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w)
