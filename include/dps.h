@@ -92,9 +92,7 @@ typedef enum {
  * weight (ties away from zero) instead of the next one towards zero, which removes the
  * shrinking bias of fast mode, and join(P, R) - the same constant still rebuilds W exactly.
  * Legal iff no b' reaches an Inf / NaN code: max|b & 0x7FFF| + 0x80 < 0x7C00 (E5M2_RN),
- * + 0x40 < 0x3F80 (E4M3_RN).  Never chosen by AUTO.  Accepted by dps_split_weights,
- * dps_reconstruct, dps_linear and dps_linear_fp8act; the grouped calls take the two
- * truncated encodings only.
+ * + 0x40 < 0x3F80 (E4M3_RN).  Never chosen by AUTO.  Accepted wherever an encoding is.
  *
  * w_fp16: device, rows*cols FP16 words.  w_persist, w_resid: device, rows*cols bytes each.
  * enc_inout: HOST int32.  On entry DPS_ENC_AUTO or one of the four encodings; on return
@@ -140,7 +138,7 @@ DPS_API dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const ui
  * For each row a in [0, A):
  *   y[a][:] = x[token_of_row ? token_of_row[a] : a][:] * W_eff(expert_of_row[a])^T
  * x: [T][K] FP16.  y: [A][N] FP16.  w_persist / w_resid: [E][N][K] bytes (w_resid may be
- * NULL in FAST mode).  enc_per_expert: HOST array of E encodings (E4M3 or E5M2), read
+ * NULL in FAST mode).  enc_per_expert: HOST array of E encodings (any of the four, never AUTO), read
  * before the call returns.  token_of_row (may be NULL) and expert_of_row: device int32[A].
  * workspace: device scratch of at least dps_moe_workspace_bytes(A, E, K) bytes, 16-byte
  * aligned, owned by the caller; its contents are overwritten (routing tables and the

@@ -265,7 +265,7 @@ int oracle_moe_linear(int mode, const int32_t* enc_per_expert, const uint16_t* x
                       const int64_t* rows_sel, int64_t n_sel, int threads) {
     if (mode != ORACLE_MODE_FAST && mode != ORACLE_MODE_FULL) return ORACLE_ERR_ARG;
     for (int32_t e = 0; e < E; ++e)
-        if (enc_per_expert[e] != ORACLE_ENC_E4M3 && enc_per_expert[e] != ORACLE_ENC_E5M2)
+        if (!known_enc(enc_per_expert[e]))
             return ORACLE_ERR_ARG;
     int bad = 0;
     int64_t count = rows_sel ? n_sel : A;

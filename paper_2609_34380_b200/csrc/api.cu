@@ -206,7 +206,7 @@ dps_status dps_moe_linear(int32_t mode, const int32_t* enc_per_expert, const voi
     const size_t need = moe_workspace_bytes(A, E, K);
     if (need == 0) return DPS_ERR_SHAPE;
     for (int32_t e = 0; e < E; ++e)
-        if (enc_per_expert[e] != DPS_ENC_E4M3 && enc_per_expert[e] != DPS_ENC_E5M2) return DPS_ERR_ENCODING;
+        if (!known_encoding(enc_per_expert[e])) return DPS_ERR_ENCODING;
     if (A == 0) return DPS_OK;
     if (!x || !expert_of_row || !w_persist || !y) return DPS_ERR_NULL;
     if (mode == DPS_MODE_FULL && !w_resid) return DPS_ERR_NULL;

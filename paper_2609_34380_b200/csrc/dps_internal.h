@@ -30,7 +30,8 @@ cudaError_t launch_decode_mma(int mode, int enc, const void* x, const uint8_t* p
 cudaError_t launch_umma_linear(int mode, int enc, const void* x, const uint8_t* p, const uint8_t* r, void* y,
                                int64_t M, int64_t N, int64_t K, int* status, cudaStream_t stream);
 
-// Grouped linear on the tensor-core path.  x_sorted: [A][K] activations grouped by expert;
+// Grouped linear on the tensor-core path.  e5m2_mask: 64 words, bit e of the first 32 set for an E5M2
+// expert, of the last 32 for a rounded nest.  x_sorted: [A][K] activations grouped by expert;
 // tiles / num_tiles / sorted_rows: device tables built by the routing pre-pass; tn: token-tile
 // width the tile list was built for (grouped_tile_tokens); max_tiles: upper bound on num_tiles.
 int grouped_tile_tokens(int64_t A, int32_t E);

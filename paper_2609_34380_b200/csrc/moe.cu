@@ -170,10 +170,14 @@ cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const i
         if (err != cudaSuccess) return err;
     }
 
-    uint32_t mask[kMaxExperts / 32];
-    for (int i = 0; i < kMaxExperts / 32; ++i) mask[i] = 0;
-    for (int e = 0; e < E; ++e)
-        if (enc_host[e] == DPS_ENC_E5M2) mask[e >> 5] |= 1u << (e & 31);
+    // 32 words of E5M2 bits, then 32 words of rounded-nest bits
+    static_assert(kMaxExperts == 1024, "the grouped kernels take two 32-word masks");
+    uint32_t mask[64];
+    for (int i = 0; i < 64; ++i) mask[i] = 0;
+    for (int e = 0; e < E; ++e) {
+        if (enc_host[e] == DPS_ENC_E5M2 || enc_host[e] == DPS_ENC_E5M2_RN) mask[e >> 5] |= 1u << (e & 31);
+        if (enc_host[e] == DPS_ENC_E4M3_RN || enc_host[e] == DPS_ENC_E5M2_RN) mask[32 + (e >> 5)] |= 1u << (e & 31);
+    }
     // an upper bound on the number of token tiles that needs no device round trip
     const int max_tiles = (int)((A + tn - 1) / tn + E);
     return launch_umma_grouped(mode, mask, w.x_sorted, p, r, y, A, N, K, E, tn, w.tiles, w.num_tiles, w.sorted_rows,
@@ -232,7 +236,7 @@ extern "C" DPS_API dps_status dps_moe_linear_static(int32_t mode, const int32_t*
     if (need == 0) return DPS_ERR_SHAPE;
     if (need > kStaticScratchBytes) return DPS_ERR_WORKSPACE;  // beyond the built-in scratch: use dps_moe_linear
     for (int32_t e = 0; e < E; ++e)
-        if (enc_per_expert[e] != DPS_ENC_E4M3 && enc_per_expert[e] != DPS_ENC_E5M2) return DPS_ERR_ENCODING;
+        if (enc_per_expert[e] < DPS_ENC_E4M3 || enc_per_expert[e] > DPS_ENC_E5M2_RN) return DPS_ERR_ENCODING;
     if (A == 0) return DPS_OK;
     if (!x || !expert_of_row || !w_persist || !y) return DPS_ERR_NULL;
     if (mode == DPS_MODE_FULL && !w_resid) return DPS_ERR_NULL;

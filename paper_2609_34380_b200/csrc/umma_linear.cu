@@ -161,7 +161,8 @@ struct GroupedParams {
     const int4* tiles;
     const int32_t* num_tiles;
     const int32_t* sorted_rows;   // sorted position -> caller's row id
-    uint32_t e5m2[32];            // bit e set: expert e is E5M2
+    uint32_t e5m2[32];            // bit e set: expert e is E5M2 (truncated or rounded)
+    uint32_t rounded[32];         // bit e set: expert e is a rounded nest (full mode only; fast mode reads P alike)
 };
 
 struct UmmaParams {
@@ -353,6 +354,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     int tile_tokens = TN;            // valid token columns of the tile (grouped)
     int plane_row0 = n0;             // first plane row of the tile in the [E * N][K] view
     bool e5m2 = (ENC == kEncE5M2);
+    bool rounded = false;         // grouped launches: this tile's expert is a rounded nest (full mode)
     if (GROUPED) {
         grid_dependency_wait();      // the tile list comes from the routing pre-pass
         if ((int)blockIdx.y >= *gp.num_tiles) return;
@@ -361,6 +363,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         tile_tokens = t.z;
         plane_row0 = t.x * prm.N + n0;
         e5m2 = (gp.e5m2[t.x >> 5] >> (t.x & 31)) & 1u;
+        rounded = FULL && ((gp.rounded[t.x >> 5] >> (t.x & 31)) & 1u);
     }
     // UMMA N of this tile.  A grouped tile multiplies only the token columns it has (rounded up to
     // 16): at 64-96 tokens per expert a fast-mode MoE layer sits at the ridge between HBM and the
@@ -602,7 +605,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2)) {
             // encoding known only at run time (one per expert): uniform branch per CTA
             ZipState zst;
-            ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
+            if (FULL && rounded)
+                ok = e5m2 ? zip_blocks<kEncE5M2R, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3R, FULL, TN, RB>(zc, zst);
+            else
+                ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
         } else {
             ZipState zst;
             ok = zip_blocks<ENC, FULL, TN, RB>(zc, zst);
@@ -763,6 +769,7 @@ struct TileCoords {
     int n0, m0, tile_tokens, plane_row0;
     int parts;   // 1, 2 or 4: this work item covers TN / parts token columns (activation box of that height)
     bool e5m2;
+    bool rounded;   // grouped launches, full mode: the expert is a rounded nest
 };
 
 // Work item `step` of this CTA: whole tiles blockIdx.x + step * gridDim.x below `t_main`, then ONE
@@ -823,12 +830,14 @@ __device__ __forceinline__ TileCoords tile_coords(int lin, int part, int parts, 
     t.tile_tokens = min(TN / t.parts, prm.M - t.m0);   // may be <= 0 for a piece past the last token: skipped
     t.plane_row0 = t.n0;
     t.e5m2 = (ENC == kEncE5M2);
+    t.rounded = false;
     if (GROUPED) {
         const int4 g = gp.tiles[tok_tile];
         t.m0 = g.y;
         t.tile_tokens = g.z;
         t.plane_row0 = g.x * prm.N + t.n0;
         t.e5m2 = (gp.e5m2[g.x >> 5] >> (g.x & 31)) & 1u;
+        t.rounded = (gp.rounded[g.x >> 5] >> (g.x & 31)) & 1u;
     }
     return t;
 }
@@ -1020,7 +1029,9 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
             if (GROUPED && zt < t.tile_tokens) s_rows[zt] = gp.sorted_rows[t.m0 + zt];
             if (ok) {
                 if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2))
-                    ok = t.e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
+                    ok = (FULL && t.rounded)
+                             ? (t.e5m2 ? zip_blocks<kEncE5M2R, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3R, FULL, TN, RB>(zc, zst))
+                             : (t.e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst));
                 else
                     ok = zip_blocks<ENC, FULL, TN, RB>(zc, zst);
             }
@@ -1694,7 +1705,10 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     gp.tiles = static_cast<const int4*>(tiles);
     gp.num_tiles = num_tiles;
     gp.sorted_rows = sorted_rows;
-    for (int i = 0; i < 32; ++i) gp.e5m2[i] = e5m2_mask[i];
+    for (int i = 0; i < 32; ++i) {   // the caller's array holds the E5M2 bits, then the rounded-nest bits
+        gp.e5m2[i] = e5m2_mask[i];
+        gp.rounded[i] = FULL ? e5m2_mask[32 + i] : 0u;
+    }
     if constexpr (kCtasPerSm == 1 && TN % kEpiChunkCols == 0) {
         const int64_t upper = ((N + kTileRows * RB - 1) / (kTileRows * RB)) * max_tiles;
         if (use_persistent(upper))

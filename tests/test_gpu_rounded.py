@@ -95,7 +95,7 @@ def test_fast_mode_error_shrinks_on_llama_o_projection():
     assert err[dps.DPS_ENC_E4M3_RN] < 0.8 * err[dps.DPS_ENC_E4M3]
 
 
-def test_fp8_activation_fast_mode_and_grouped_calls():
+def test_fp8_activation_fast_mode():
     N, K, M = 264, 528, 40
     w = workloads.weights(N, K, 31, device=DEV)
     x = workloads.activations(M, K, 32, device=DEV)
@@ -106,10 +106,39 @@ def test_fp8_activation_fast_mode_and_grouped_calls():
         ref = oracle.linear_fp8act(enc, to_np_bytes(q), scale.cpu().numpy(), to_np_bytes(p), threads=4)
         assert_close_to_oracle(y, ref, f"fp8act rounded enc={enc}")
         assert torch.equal(y, dps.dps_linear_fp8act(base, q, scale, p))
-    # the grouped calls take the truncated encodings only
-    P = torch.zeros((2, 128, 64), dtype=torch.uint8, device=DEV)
-    xs = workloads.activations(4, 64, 1, device=DEV)
-    eor = torch.tensor([0, 1, 0, 1], dtype=torch.int32, device=DEV)
-    with pytest.raises(dps.DpsError) as e:
-        dps.dps_moe_linear(dps.DPS_MODE_FAST, [dps.DPS_ENC_E4M3_RN, dps.DPS_ENC_E4M3], xs, None, eor, P, None)
-    assert e.value.status == dps.binding.DPS_ERR_ENCODING
+
+
+def test_grouped_linear_with_rounded_and_truncated_experts():
+    """Experts of all four encodings in one call; one expert with a second token tile, one empty."""
+    E, N, K, T = 5, 392, 528, 140
+    req = [dps.DPS_ENC_E4M3_RN, dps.DPS_ENC_E5M2, dps.DPS_ENC_E5M2_RN, dps.DPS_ENC_E4M3, dps.DPS_ENC_E4M3_RN]
+    ps, rs, encs = [], [], []
+    for e in range(E):
+        w = workloads.weights(N, K, 150 + e, device=DEV)
+        p, r, enc = dps.dps_split_weights(w, req[e])
+        ps.append(p), rs.append(r), encs.append(enc)
+    assert encs == req
+    p, r = torch.stack(ps), torch.stack(rs)
+    x = workloads.activations(T, K, 160, device=DEV)
+    tor, eor = workloads.top2_routing(T, E, 170)
+    eor[eor == E - 1] = 0                         # the last expert stays empty, expert 0 gets two shares
+    tor_d, eor_d = torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV)
+    for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):
+        y = dps.dps_moe_linear(mode, encs, x, tor_d, eor_d, p, r if mode else None)
+        ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r), threads=8)
+        assert rc == oracle.OK
+        assert_close_to_oracle(y, ref, f"grouped rounded mode={mode}")
+        y_static = torch.empty_like(y)
+        dps.dps_moe_linear_static(mode, encs, x, tor_d, eor_d, p, r if mode else None, y_static)
+        assert torch.equal(y, y_static)
+    # full mode: the same outputs as with every expert stored as its truncated sibling
+    base = {dps.DPS_ENC_E4M3_RN: dps.DPS_ENC_E4M3, dps.DPS_ENC_E5M2_RN: dps.DPS_ENC_E5M2}
+    ps2, rs2, encs2 = [], [], []
+    for e in range(E):
+        w = workloads.weights(N, K, 150 + e, device=DEV)
+        p2, r2, enc2 = dps.dps_split_weights(w, base.get(req[e], req[e]))
+        ps2.append(p2), rs2.append(r2), encs2.append(enc2)
+    y_rn = dps.dps_moe_linear(dps.DPS_MODE_FULL, encs, x, tor_d, eor_d, p, r)
+    y_tr = dps.dps_moe_linear(dps.DPS_MODE_FULL, encs2, x, tor_d, eor_d, torch.stack(ps2), torch.stack(rs2))
+    assert torch.equal(y_rn, y_tr)
+    assert dps.dps_stream_status() == dps.DPS_OK
