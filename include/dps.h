@@ -76,7 +76,8 @@ typedef enum {
     DPS_ENC_E4M3 = 1,
     DPS_ENC_E5M2 = 2,
     DPS_ENC_E4M3_RN = 3, /* rounded nests, see below */
-    DPS_ENC_E5M2_RN = 4
+    DPS_ENC_E5M2_RN = 4,
+    DPS_ENC_AUTO_RN = 5  /* dps_split_weights only: AUTO's rule, answering with a rounded nest */
 } dps_encoding;
 
 /*
@@ -92,10 +93,12 @@ typedef enum {
  * weight (ties away from zero) instead of the next one towards zero, which removes the
  * shrinking bias of fast mode, and join(P, R) - the same constant still rebuilds W exactly.
  * Legal iff no b' reaches an Inf / NaN code: max|b & 0x7FFF| + 0x80 < 0x7C00 (E5M2_RN),
- * + 0x40 < 0x3F80 (E4M3_RN).  Never chosen by AUTO.  Accepted wherever an encoding is.
+ * + 0x40 < 0x3F80 (E4M3_RN).  Never chosen by AUTO; DPS_ENC_AUTO_RN chooses between them by
+ * AUTO's rule (E4M3_RN iff max|w| <= 1.75, else E5M2_RN; DPS_ERR_DATA if that is not legal
+ * either, i.e. |w| >= 61440 or Inf / NaN present).  Accepted wherever an encoding is.
  *
  * w_fp16: device, rows*cols FP16 words.  w_persist, w_resid: device, rows*cols bytes each.
- * enc_inout: HOST int32.  On entry DPS_ENC_AUTO or one of the four encodings; on return
+ * enc_inout: HOST int32.  On entry DPS_ENC_AUTO, DPS_ENC_AUTO_RN or one of the four encodings; on return
  * the encoding that was used.
  *   AUTO  -> E4M3 iff every word has b[14] == 0 and max|w| <= 1.75, else E5M2.  The
  *            statistics pass needs its result on the host, so this variant SYNCHRONISES

@@ -24,6 +24,7 @@ import numpy as np
 MODE_FAST, MODE_FULL = 0, 1
 ENC_AUTO, ENC_E4M3, ENC_E5M2 = 0, 1, 2
 ENC_E4M3_RN, ENC_E5M2_RN = 3, 4          # rounded nests (an extension, see dps_oracle.c)
+ENC_AUTO_RN = 5                          # split only: the AUTO rule, answering with a rounded nest
 OK, ERR_ARG, ERR_DATA = 0, 1, 8
 
 _HERE = Path(__file__).resolve().parent
@@ -144,6 +145,8 @@ def split(w, enc: int):
     w = _words(w)
     if enc == ENC_AUTO:
         enc = select_encoding(w)
+    elif enc == ENC_AUTO_RN:                 # the same rule; an illegal answer is refused by the split below
+        enc = ENC_E4M3_RN if select_encoding(w) == ENC_E4M3 else ENC_E5M2_RN
     p = np.empty(w.shape, np.uint8)
     r = np.empty(w.shape, np.uint8)
     rc = lib().oracle_split(_ptr(w), _ptr(p), _ptr(r), w.size, enc)

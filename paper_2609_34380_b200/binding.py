@@ -15,6 +15,7 @@ import torch
 DPS_MODE_FAST, DPS_MODE_FULL = 0, 1
 DPS_ENC_AUTO, DPS_ENC_E4M3, DPS_ENC_E5M2 = 0, 1, 2
 DPS_ENC_E4M3_RN, DPS_ENC_E5M2_RN = 3, 4      # rounded nests
+DPS_ENC_AUTO_RN = 5                          # dps_split_weights only: AUTO's rule, rounded nests
 DPS_OK = 0
 DPS_ERR_NULL, DPS_ERR_SHAPE, DPS_ERR_MODE, DPS_ERR_ENCODING, DPS_ERR_ALIGN = 1, 2, 3, 4, 5
 DPS_ERR_UNSUPPORTED, DPS_ERR_CUDA, DPS_ERR_DATA, DPS_ERR_WORKSPACE = 6, 7, 8, 9

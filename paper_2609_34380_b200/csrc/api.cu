@@ -99,12 +99,13 @@ dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_
                              int32_t* enc_inout, void* cuda_stream) {
     if (enc_inout == nullptr) return DPS_ERR_NULL;
     const int32_t req = *enc_inout;
-    if (req != DPS_ENC_AUTO && !known_encoding(req)) return DPS_ERR_ENCODING;
+    if (req != DPS_ENC_AUTO && req != DPS_ENC_AUTO_RN && !known_encoding(req)) return DPS_ERR_ENCODING;
     if (rows < 0 || cols < 0 || (cols % 16) != 0) return DPS_ERR_SHAPE;
     if (rows > 0 && cols > 0 && rows > INT64_MAX / cols) return DPS_ERR_SHAPE;
     const int64_t n = rows * cols;
     if (n == 0) {
         if (req == DPS_ENC_AUTO) *enc_inout = DPS_ENC_E4M3;
+        if (req == DPS_ENC_AUTO_RN) *enc_inout = DPS_ENC_E4M3_RN;
         return DPS_OK;
     }
     if (!w_fp16 || !w_persist || !w_resid) return DPS_ERR_NULL;
@@ -130,6 +131,10 @@ dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_
             return DPS_ERR_CUDA;
         if (cudaStreamSynchronize(stream) != cudaSuccess) return DPS_ERR_CUDA;
         if (req == DPS_ENC_AUTO) enc = (maxmag <= 0x3F00u) ? DPS_ENC_E4M3 : DPS_ENC_E5M2;
+        else if (req == DPS_ENC_AUTO_RN) {
+            enc = (maxmag <= 0x3F00u) ? DPS_ENC_E4M3_RN : DPS_ENC_E5M2_RN;
+            if (enc == DPS_ENC_E5M2_RN && maxmag + 0x80u >= 0x7C00u) return DPS_ERR_DATA;
+        }
         else if (req == DPS_ENC_E4M3 && maxmag >= 0x3F80u) return DPS_ERR_DATA;
         else if (req == DPS_ENC_E4M3_RN && maxmag + 0x40u >= 0x3F80u) return DPS_ERR_DATA;
         else if (req == DPS_ENC_E5M2_RN && maxmag + 0x80u >= 0x7C00u) return DPS_ERR_DATA;

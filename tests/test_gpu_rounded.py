@@ -142,3 +142,22 @@ def test_grouped_linear_with_rounded_and_truncated_experts():
     y_tr = dps.dps_moe_linear(dps.DPS_MODE_FULL, encs2, x, tor_d, eor_d, torch.stack(ps2), torch.stack(rs2))
     assert torch.equal(y_rn, y_tr)
     assert dps.dps_stream_status() == dps.DPS_OK
+
+
+def test_auto_rule_answers_with_a_rounded_nest():
+    w = workloads.weights(16, 64, 9, device=DEV)
+    p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO_RN)
+    assert enc == dps.DPS_ENC_E4M3_RN
+    p_ref, r_ref, enc_ref = oracle.split(to_np_words(w), oracle.ENC_AUTO_RN)
+    assert enc_ref == enc and np.array_equal(to_np_bytes(p), p_ref) and np.array_equal(to_np_bytes(r), r_ref)
+    w2 = workloads.with_outlier(w)
+    p, r, enc = dps.dps_split_weights(w2, dps.DPS_ENC_AUTO_RN)
+    assert enc == dps.DPS_ENC_E5M2_RN
+    assert torch.equal(dps.dps_reconstruct(p, r, enc).view(torch.int16), w2.view(torch.int16))
+    with pytest.raises(dps.DpsError) as e:
+        dps.dps_split_weights(workloads.with_outlier(w, 61440.0), dps.DPS_ENC_AUTO_RN)
+    assert e.value.status == dps.binding.DPS_ERR_DATA
+    # AUTO_RN names no stored format: the other calls refuse it
+    with pytest.raises(dps.DpsError) as e:
+        dps.dps_reconstruct(p, r, dps.DPS_ENC_AUTO_RN)
+    assert e.value.status == dps.binding.DPS_ERR_ENCODING

@@ -129,3 +129,15 @@ def test_linear_full_mode_is_unchanged_and_fast_mode_uses_the_rounded_weights():
         # closer to the full-mode result than the truncated nest's fast mode
         fast_trunc = oracle.linear(oracle.MODE_FAST, base, xw, pb, rb)
         assert np.abs(fast - full).mean() < np.abs(fast_trunc - full).mean()
+
+
+def test_auto_rule_answers_with_a_rounded_nest():
+    w = workloads.weights(8, 64, 9)
+    words = workloads.as_words(w)
+    _, _, enc = oracle.split(words, oracle.ENC_AUTO_RN)
+    assert enc == oracle.ENC_E4M3_RN and oracle.select_encoding(words) == oracle.ENC_E4M3
+    _, _, enc = oracle.split(workloads.as_words(workloads.with_outlier(w)), oracle.ENC_AUTO_RN)
+    assert enc == oracle.ENC_E5M2_RN
+    assert oracle.half_to_double(0x7B80) == 61440.0                       # the first magnitude no rounded nest can hold
+    with pytest.raises(oracle.OracleError):
+        oracle.split(workloads.as_words(workloads.with_outlier(w, 61440.0)), oracle.ENC_AUTO_RN)
