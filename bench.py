@@ -510,7 +510,14 @@ def detail_rows(dps, workloads, torch, dev, peaks):
             else:
                 rn[f"qkv_M2048_full_{label}_TFLOP/s"] = 4 * 2 * M * n * k / (ms * 1e-3) / 1e12
             del x, y
-        del pl
+        # what the rounded nest buys: distance of the fast-mode output from the full-mode one (8 tokens)
+        x = workloads.activations(8, k, 3001, device=dev)
+        p, r, e = pl[0]
+        y_full = dps.dps_linear(dps.DPS_MODE_FULL, e, x, p, r).double()
+        y_fast = dps.dps_linear(dps.DPS_MODE_FAST, e, x, p, None).double()
+        rn[f"qkv_M8_fast_vs_full_mean_abs_diff_{label}"] = (y_fast - y_full).abs().mean().item()
+        rn[f"qkv_M8_fast_over_full_projection_{label}"] = ((y_fast * y_full).sum() / (y_full * y_full).sum()).item()
+        del x, y_full, y_fast, pl
     rn["what"] = ("Llama-7B QKV, 4 weight copies in rotation, full mode, E4M3 nest against its rounded variant "
                   "(fast mode runs the same kernels on either plane)")
     out["rounded_nest"] = rn
