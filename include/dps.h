@@ -95,7 +95,9 @@ typedef enum {
  * Legal iff no b' reaches an Inf / NaN code: max|b & 0x7FFF| + 0x80 < 0x7C00 (E5M2_RN),
  * + 0x40 < 0x3F80 (E4M3_RN).  Never chosen by AUTO; DPS_ENC_AUTO_RN chooses between them by
  * AUTO's rule (E4M3_RN iff max|w| <= 1.75, else E5M2_RN; DPS_ERR_DATA if that is not legal
- * either, i.e. |w| >= 61440 or Inf / NaN present).  Accepted wherever an encoding is.
+ * either, i.e. |w| >= 61440 or Inf / NaN present).  Accepted wherever an encoding is.  In a legal
+ * rounded pair a zero P byte never meets a zero R byte; the linear kernels read such a pair (their
+ * own padding) as a zero weight.
  *
  * w_fp16: device, rows*cols FP16 words.  w_persist, w_resid: device, rows*cols bytes each.
  * enc_inout: HOST int32.  On entry DPS_ENC_AUTO, DPS_ENC_AUTO_RN or one of the four encodings; on return
@@ -108,7 +110,8 @@ typedef enum {
  *            planes untouched.
  *   E5M2  -> always legal, never synchronises.
  *   E4M3_RN, E5M2_RN -> checked like E4M3 (synchronise; DPS_ERR_DATA if not legal).
- * rows*cols == 0 returns DPS_OK (AUTO then reports E4M3).  cols must be a multiple of 16.
+ * rows*cols == 0 returns DPS_OK (AUTO then reports E4M3, AUTO_RN E4M3_RN).  cols must be a
+ * multiple of 16.
  */
 DPS_API dps_status dps_split_weights(const void* w_fp16, uint8_t* w_persist, uint8_t* w_resid,
                              int64_t rows, int64_t cols, int32_t* enc_inout, void* cuda_stream);
