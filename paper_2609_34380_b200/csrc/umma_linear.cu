@@ -36,6 +36,7 @@
 #include "bits.cuh"
 #include "dps_internal.h"
 #include "sm100.cuh"
+#include "tensor_map.h"
 
 namespace dps {
 
@@ -1163,10 +1164,6 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
 
 // ---- host side ---------------------------------------------------------------------------------
 
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 // Tuning knob: DPS_PAIR_MIN=<depth> sets the (even) ring depth from which two stages are filled at a
 // time, so that two boxes cover 256 adjacent bytes of every weight row.  Off by default: with rings
 // of 5-7 stages it was measured equal or slower (up to 20 % on a 6-deep full-mode ring) than
@@ -1186,31 +1183,6 @@ int forced_split() {
         return e ? atoi(e) : 0;
     }();
     return v;
-}
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// 2-D row-major tensor [rows][cols] of `elem_bytes`-sized elements, tiles of box_rows x box_cols.
-bool make_map_2d(CUtensorMap* map, const void* base, CUtensorMapDataType dt, int elem_bytes, uint64_t rows,
-                 uint64_t cols, uint32_t box_rows, uint32_t box_cols, CUtensorMapSwizzle swizzle) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
-    const cuuint32_t box[2] = {box_cols, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // K split for a launch of `tiles` output tiles.  capacity[s] = CTAs that can be resident at once
