@@ -180,7 +180,8 @@ DPS_API size_t dps_moe_workspace_bytes(int64_t A, int32_t E, int64_t K);
  *     the library until the process exits.  A problem whose dps_moe_workspace_bytes(A, E, K) exceeds
  *     it is rejected with DPS_ERR_WORKSPACE and nothing is enqueued; use dps_moe_linear then.
  *   - The first call on each device looks up the array's device address (a one-time, host-side
- *     set-up step).  Make that first call outside any stream capture.
+ *     set-up step).  Make that first call outside any stream capture.  If the look-up fails the
+ *     call returns DPS_ERR_CUDA and keeps nothing: a later call simply tries again.
  *   - All calls on a device share the one array and it keeps whatever the last call left in it.
  *     Nothing in it has to start at zero: every call rewrites all the tables it reads.  Two calls
  *     whose kernels can overlap on the GPU (different streams without an ordering between them)
@@ -196,8 +197,8 @@ DPS_API dps_status dps_moe_linear_static(int32_t mode, const int32_t* enc_per_ex
                                          void* cuda_stream);
 
 /*
- * Fast mode with FP8 activations (paper: "Persistent Region" paragraph -- FP8 execution can "double
- * peak tensor-core throughput with hardware support").  The persistent plane is fed to the FP8
+ * Fast mode with FP8 activations (paper: "Persistent Region" paragraph, which notes that FP8
+ * execution can raise the tensor-core peak where the hardware supports it).  The persistent plane is fed to the FP8
  * tensor cores as it is; the activations are quantised per token:
  *   scale[m] = max_k |x[m][k]| / 448 (1 for an all-zero token),
  *   x_fp8[m][k] = E4M3(x[m][k] / scale[m]), round to nearest even, saturating (both in binary32),
@@ -238,6 +239,16 @@ DPS_API dps_status dps_restore_residual(uint8_t* w_resid, const uint8_t* backup_
  * DPS_OK, DPS_ERR_DATA (a kernel skipped a row with a bad index) or DPS_ERR_CUDA.
  */
 DPS_API dps_status dps_stream_status(void* cuda_stream);
+
+/*
+ * Diagnostic: exercises the bounded device-side wait that every pipeline of the tensor-core kernels
+ * uses.  One warp waits, for at most limit_ns nanoseconds (1 .. 1e9), on a barrier that nothing
+ * ever signals; when the limit passes it sets the status word and returns, exactly as a kernel does
+ * whose copy never arrives.  Afterwards dps_stream_status() reports DPS_ERR_CUDA once, and the
+ * device and the library remain fully usable.  Nothing faults, traps or spins without a limit.
+ * (No counterpart in the paper: it tests this library's own failure handling.)
+ */
+DPS_API dps_status dps_debug_wait_timeout(uint64_t limit_ns, void* cuda_stream);
 
 /* Number of kernel launches this process has enqueued through the library so far. */
 DPS_API int64_t dps_launch_count(void);

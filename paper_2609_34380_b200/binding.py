@@ -38,6 +38,7 @@ ABI = {
     "dps_backup_residual": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t, ctypes.c_size_t, _vp]),
     "dps_restore_residual": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t, ctypes.c_size_t, _vp]),
     "dps_stream_status": (ctypes.c_int, [_vp]),
+    "dps_debug_wait_timeout": (ctypes.c_int, [ctypes.c_uint64, _vp]),
     "dps_launch_count": (_i64, []),
     "dps_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "dps_version": (ctypes.c_int, []),
@@ -258,6 +259,12 @@ def dps_restore_residual(w_resid: torch.Tensor, backup_host: torch.Tensor, chunk
 def dps_stream_status(stream=None) -> int:
     """Synchronise the stream; return and clear the device status word."""
     return int(library().dps_stream_status(_stream(stream)))
+
+
+def dps_debug_wait_timeout(limit_ns: int, stream=None) -> None:
+    """Launches the self-test of the bounded device-side wait: one warp waits `limit_ns` nanoseconds for a
+    barrier nobody signals, then sets the status word (dps_stream_status reports DPS_ERR_CUDA once)."""
+    _check(library().dps_debug_wait_timeout(int(limit_ns), _stream(stream)), "dps_debug_wait_timeout")
 
 
 def dps_launch_count() -> int:

@@ -73,21 +73,5 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
     return LIB
 
 
-def build_microbench() -> list:
-    """Compile the stand-alone hardware microbenchmarks under microbench/ (not needed by the library)."""
-    out = []
-    for src in sorted((PKG / "microbench").glob("*.cu")):
-        exe = src.with_suffix("")
-        cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-o", str(exe), str(src)]
-        res = subprocess.run(cmd, capture_output=True, text=True)
-        if res.returncode != 0:
-            raise RuntimeError(f"nvcc failed for {src.name}:\n{res.stdout}\n{res.stderr}")
-        out.append(exe)
-    return out
-
-
 if __name__ == "__main__":
-    if "--microbench" in sys.argv:
-        print(*build_microbench(), sep="\n")
-    else:
-        print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_library(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -5,6 +5,8 @@
 #include <cstring>
 #include <mutex>
 
+#include "sm100.cuh"
+
 #include "bits.cuh"
 #include "dps_internal.h"
 
@@ -12,12 +14,25 @@ namespace dps {
 
 namespace {
 
-constexpr int kMaxDevices = 64;
-
 // Per-device words that kernels write: the status word (data-dependent errors) and the
 // scratch word of the load-time magnitude statistic.
 __device__ int g_status_word;
 __device__ unsigned g_stat_word;
+
+// Self-test of the bounded device-side waits: ONE warp initialises an mbarrier that nobody will ever
+// arrive on and waits for it with the given limit -- the same wait (and the same reaction: set the
+// status word, give up, return) as every pipeline wait in the tensor-core kernels.  No copy is in
+// flight, no tensor memory is held, no other CTA is involved.
+__global__ void wait_timeout_selftest_kernel(unsigned long long limit_ns, int* status) {
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        sm100::mbar_init(sm100::smem_u32(&bar), 1);
+        sm100::fence_barrier_init();
+    }
+    __syncwarp();
+    if (!sm100::mbar_wait_limit(sm100::smem_u32(&bar), 0, limit_ns) && threadIdx.x == 0)
+        atomicExch(status, (int)DPS_ERR_CUDA);
+}
 
 std::atomic<int64_t> g_launches{0};
 std::mutex g_stat_mutex;  // the statistic word is shared by all AUTO / checked-E4M3 splits
@@ -70,6 +85,36 @@ dps_status check_device(DeviceInfo*& d) {
 }  // namespace
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+dps_status check_moe_args(int32_t mode, const int32_t* enc_per_expert, const void* x, const int32_t* token_of_row,
+                          const int32_t* expert_of_row, const uint8_t* w_persist, const uint8_t* w_resid, const void* y,
+                          int64_t A, int64_t T, int64_t N, int64_t K, int32_t E, bool* empty) {
+    *empty = false;
+    if (mode != DPS_MODE_FAST && mode != DPS_MODE_FULL) return DPS_ERR_MODE;
+    if (A < 0 || T < 0 || N <= 0 || K <= 0 || E <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
+    if (A > ((int64_t)1 << 30) || T > ((int64_t)1 << 30) || N >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31))
+        return DPS_ERR_SHAPE;
+    // the kernels address plane rows of all experts with 32-bit coordinates
+    if ((int64_t)E * N >= ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
+    if (!enc_per_expert) return DPS_ERR_NULL;
+    if (moe_workspace_bytes(A, E, K) == 0) return DPS_ERR_SHAPE;
+    for (int32_t e = 0; e < E; ++e) {
+        const int32_t enc = enc_per_expert[e];
+        if (enc != DPS_ENC_E4M3 && enc != DPS_ENC_E5M2 && enc != DPS_ENC_E4M3_RN && enc != DPS_ENC_E5M2_RN)
+            return DPS_ERR_ENCODING;
+    }
+    if (A == 0) {
+        *empty = true;
+        return DPS_OK;
+    }
+    if (!x || !expert_of_row || !w_persist || !y) return DPS_ERR_NULL;
+    if (mode == DPS_MODE_FULL && !w_resid) return DPS_ERR_NULL;
+    if (!aligned16(x) || !aligned16(w_persist) || !aligned16(y)) return DPS_ERR_ALIGN;
+    if (mode == DPS_MODE_FULL && !aligned16(w_resid)) return DPS_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(expert_of_row) & 3u) || (reinterpret_cast<uintptr_t>(token_of_row) & 3u))
+        return DPS_ERR_ALIGN;
+    return DPS_OK;
+}
 
 dps_status device_status_word(int** status) {
     DeviceInfo* d = nullptr;
@@ -168,7 +213,7 @@ dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w
     if (mode != DPS_MODE_FAST && mode != DPS_MODE_FULL) return DPS_ERR_MODE;
     if (!known_encoding(enc)) return DPS_ERR_ENCODING;
     if (M < 0 || N <= 0 || K <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
-    if (N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31) || M > ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
+    if (N >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31) || M >= ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
     if (M == 0) return DPS_OK;
     if (!x || !w_persist || !y) return DPS_ERR_NULL;
     if (mode == DPS_MODE_FULL && !w_resid) return DPS_ERR_NULL;
@@ -191,7 +236,7 @@ dps_status dps_linear(int32_t mode, int32_t enc, const void* x, const uint8_t* w
     if (path == 1) err = launch_gemv(mode, enc, x, w_persist, r, y, M, N, K, stream);
     else if (path == 2) err = launch_umma_linear(mode, enc, x, w_persist, r, y, M, N, K, d->status, stream);
     else if (path == 3 || M <= 8 || (M <= 16 && stream_mid)) {
-        if (M > 32) return DPS_ERR_UNSUPPORTED;
+        if (M > 16) return DPS_ERR_UNSUPPORTED;      // (only reachable with DPS_FORCE_PATH=stream)
         err = launch_decode_mma(mode, enc, x, w_persist, r, y, M, N, K, stream);
     } else err = launch_umma_linear(mode, enc, x, w_persist, r, y, M, N, K, d->status, stream);
     return err == cudaSuccess ? DPS_OK : DPS_ERR_CUDA;
@@ -203,22 +248,11 @@ dps_status dps_moe_linear(int32_t mode, const int32_t* enc_per_expert, const voi
                           const int32_t* expert_of_row, const uint8_t* w_persist, const uint8_t* w_resid, void* y,
                           int64_t A, int64_t T, int64_t N, int64_t K, int32_t E, void* workspace,
                           size_t workspace_bytes, void* cuda_stream) {
-    if (mode != DPS_MODE_FAST && mode != DPS_MODE_FULL) return DPS_ERR_MODE;
-    if (A < 0 || T < 0 || N <= 0 || K <= 0 || E <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
-    if (A > ((int64_t)1 << 30) || T > ((int64_t)1 << 30) || N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31))
-        return DPS_ERR_SHAPE;
-    if (!enc_per_expert) return DPS_ERR_NULL;
+    bool empty = false;
+    const dps_status ok = check_moe_args(mode, enc_per_expert, x, token_of_row, expert_of_row, w_persist, w_resid, y, A, T,
+                                         N, K, E, &empty);
+    if (ok != DPS_OK || empty) return ok;
     const size_t need = moe_workspace_bytes(A, E, K);
-    if (need == 0) return DPS_ERR_SHAPE;
-    for (int32_t e = 0; e < E; ++e)
-        if (!known_encoding(enc_per_expert[e])) return DPS_ERR_ENCODING;
-    if (A == 0) return DPS_OK;
-    if (!x || !expert_of_row || !w_persist || !y) return DPS_ERR_NULL;
-    if (mode == DPS_MODE_FULL && !w_resid) return DPS_ERR_NULL;
-    if (!aligned16(x) || !aligned16(w_persist) || !aligned16(y)) return DPS_ERR_ALIGN;
-    if (mode == DPS_MODE_FULL && !aligned16(w_resid)) return DPS_ERR_ALIGN;
-    if ((reinterpret_cast<uintptr_t>(expert_of_row) & 3u) || (reinterpret_cast<uintptr_t>(token_of_row) & 3u))
-        return DPS_ERR_ALIGN;
     if (!workspace || !aligned16(workspace) || workspace_bytes < need) return DPS_ERR_WORKSPACE;
     DeviceInfo* d;
     dps_status st = check_device(d);
@@ -245,7 +279,7 @@ dps_status dps_stream_status(void* cuda_stream) {
 
 dps_status dps_quantize_activations(const void* x, uint8_t* x_fp8, float* scale, int64_t M, int64_t K,
                                     void* cuda_stream) {
-    if (M < 0 || K <= 0 || (K % 16) != 0 || M > ((int64_t)1 << 31) || K > ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
+    if (M < 0 || K <= 0 || (K % 16) != 0 || M >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
     if (M == 0) return DPS_OK;
     if (!x || !x_fp8 || !scale) return DPS_ERR_NULL;
     if (!aligned16(x) || !aligned16(x_fp8)) return DPS_ERR_ALIGN;
@@ -263,7 +297,7 @@ dps_status dps_linear_fp8act(int32_t enc, const uint8_t* x_fp8, const float* sca
     if (!known_encoding(enc)) return DPS_ERR_ENCODING;
     enc = base_enc(enc);   // the persistent byte of a rounded nest is an FP8 value like any other
     if (M < 0 || N <= 0 || K <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
-    if (N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31) || M > ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
+    if (N >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31) || M >= ((int64_t)1 << 31)) return DPS_ERR_SHAPE;
     if (M == 0) return DPS_OK;
     if (!x_fp8 || !scale || !w_persist || !y) return DPS_ERR_NULL;
     if (!aligned16(x_fp8) || !aligned16(w_persist) || !aligned16(y)) return DPS_ERR_ALIGN;
@@ -300,6 +334,16 @@ dps_status dps_backup_residual(const uint8_t* w_resid, uint8_t* backup_host, siz
 dps_status dps_restore_residual(uint8_t* w_resid, const uint8_t* backup_host, size_t bytes, size_t chunk_bytes,
                                 void* cuda_stream) {
     return chunked_copy(w_resid, backup_host, bytes, chunk_bytes, cudaMemcpyHostToDevice, cuda_stream);
+}
+
+dps_status dps_debug_wait_timeout(uint64_t limit_ns, void* cuda_stream) {
+    if (limit_ns == 0 || limit_ns > 1000000000ull) return DPS_ERR_SHAPE;   // at most one second
+    DeviceInfo* d;
+    dps_status st = check_device(d);
+    if (st != DPS_OK) return st;
+    wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(limit_ns, d->status);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? DPS_OK : DPS_ERR_CUDA;
 }
 
 int64_t dps_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -1,5 +1,4 @@
-// Decode linear layer for a handful of tokens (up to 16; NT = 4 for up to 32 exists for comparison):
-// a register-streaming kernel.
+// Decode linear layer for a handful of tokens (up to 16): a register-streaming kernel.
 //
 // Paper: "Scheduler: Dual-Precision Execution" -- fast mode streams the FP8 tensor only, full mode
 // streams the FP8 and the residual tensor and rebuilds the FP16 weights during computation.  With
@@ -293,8 +292,7 @@ cudaError_t launch_enc(const __half* x, const uint8_t* p, const uint8_t* r, __ha
         if (M <= 16) return launch_one<ENC, FULL, 2, 2 * U, false>(x, p, r, y, M, N, K, stream);
     }
     if (M <= 8) return launch_one<ENC, FULL, 1, U, false>(x, p, r, y, M, N, K, stream);
-    if (M <= 16) return launch_one<ENC, FULL, 2, U, false>(x, p, r, y, M, N, K, stream);
-    return launch_one<ENC, FULL, 4, U, false>(x, p, r, y, M, N, K, stream);
+    return launch_one<ENC, FULL, 2, U, false>(x, p, r, y, M, N, K, stream);   // (callers never pass more than 16 tokens)
 }
 
 }  // namespace

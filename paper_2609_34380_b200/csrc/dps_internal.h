@@ -4,9 +4,32 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/dps.h"
 
 namespace dps {
+
+// One-time set-up that must happen once PER DEVICE (function attributes, occupancy queries): keyed by
+// the current device's ordinal, safe against concurrent first calls.  The error of a failed set-up is
+// kept and returned to every later caller on that device.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+    std::once_flag once[kMaxDevices];
+    cudaError_t err[kMaxDevices] = {};
+    // Runs f() the first time the current device is seen; returns its (cached) result.  *device, if
+    // given, receives the ordinal.
+    template <typename F>
+    cudaError_t run(F f, int* device = nullptr) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        if (device) *device = dev;
+        std::call_once(once[dev], [&] { err[dev] = f(); });
+        return err[dev];
+    }
+};
 
 // Every launcher enqueues on `stream`, never synchronises and returns the CUDA error of the
 // launch.  `status` is the address of the current device's status word.
@@ -53,6 +76,12 @@ cudaError_t launch_moe(int mode, const int32_t* enc_host, const void* x, const i
                        const int32_t* expert_of_row, const uint8_t* p, const uint8_t* r, void* y, int64_t A,
                        int64_t T, int64_t N, int64_t K, int32_t E, void* workspace, int* status,
                        cudaStream_t stream);
+
+// Host-side checks shared by dps_moe_linear and dps_moe_linear_static (everything but the workspace).
+// *empty is set when there is nothing to do (A == 0) and the pointers were therefore not looked at.
+dps_status check_moe_args(int32_t mode, const int32_t* enc_per_expert, const void* x, const int32_t* token_of_row,
+                          const int32_t* expert_of_row, const uint8_t* w_persist, const uint8_t* w_resid, const void* y,
+                          int64_t A, int64_t T, int64_t N, int64_t K, int32_t E, bool* empty);
 
 // Checks that the current device can run the kernels and returns the address of its status word.
 dps_status device_status_word(int** status);

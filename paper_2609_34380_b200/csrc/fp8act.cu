@@ -359,13 +359,13 @@ namespace {
 template <int kTokens>
 cudaError_t launch_fp8_tokens(int enc, const uint8_t* q, const float* scale, const uint8_t* p, void* y, int64_t M, int64_t N,
                               int64_t K, int* status, cudaStream_t stream) {
-    static bool configured = false;
+    static PerDeviceOnce setup;     // per instantiation and per device
     const size_t smem = (size_t)stages_fp8(kTokens) * stage_bytes_fp8(kTokens) + kEpiBytes + 1024;
     auto kernel = fp8act_linear_kernel<kTokens>;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    {
+        const cudaError_t e = setup.run(
+            [&] { return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); });
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     CUtensorMap mp, mx;
     if (!make_byte_map_sw128(&mp, p, (uint64_t)N, (uint64_t)K, kRows) ||

@@ -196,26 +196,28 @@ namespace {
 constexpr size_t kStaticScratchBytes = (size_t)DPS_MOE_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_moe_static_scratch[kStaticScratchBytes];
 
-struct StaticScratch {
-    std::once_flag once;
-    cudaError_t err = cudaSuccess;
-    unsigned char* ptr = nullptr;
-};
-StaticScratch g_static_scratch[64];
+// Device address of the array, per device.  Only a successful look-up is kept: a failed one (made
+// inside a stream capture, say) is tried again by the next call.
+std::mutex g_static_scratch_mutex;
+unsigned char* g_static_scratch_ptr[kMaxDevices] = {};
 
 cudaError_t static_scratch_address(unsigned char** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    StaticScratch& s = g_static_scratch[dev];
-    std::call_once(s.once, [&] {
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (g_static_scratch_ptr[dev] == nullptr) {
         unsigned char* ptr = nullptr;
-        s.err = cudaGetSymbolAddress((void**)&ptr, g_moe_static_scratch);
-        s.ptr = (s.err == cudaSuccess) ? ptr : nullptr;
-    });
-    *out = s.ptr;
-    return s.err;
+        e = cudaGetSymbolAddress((void**)&ptr, g_moe_static_scratch);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();   // leave no sticky error behind: the next call tries again
+            return e;
+        }
+        g_static_scratch_ptr[dev] = ptr;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return cudaSuccess;
 }
 
 }  // namespace
@@ -227,23 +229,12 @@ extern "C" DPS_API dps_status dps_moe_linear_static(int32_t mode, const int32_t*
                                                     int64_t A, int64_t T, int64_t N, int64_t K, int32_t E,
                                                     void* cuda_stream) {
     using namespace dps;
-    if (mode != DPS_MODE_FAST && mode != DPS_MODE_FULL) return DPS_ERR_MODE;
-    if (A < 0 || T < 0 || N <= 0 || K <= 0 || E <= 0 || (K % 16) != 0 || (N % 8) != 0) return DPS_ERR_SHAPE;
-    if (A > ((int64_t)1 << 30) || T > ((int64_t)1 << 30) || N > ((int64_t)1 << 31) || K > ((int64_t)1 << 31))
-        return DPS_ERR_SHAPE;
-    if (!enc_per_expert) return DPS_ERR_NULL;
-    const size_t need = moe_workspace_bytes(A, E, K);
-    if (need == 0) return DPS_ERR_SHAPE;
-    if (need > kStaticScratchBytes) return DPS_ERR_WORKSPACE;  // beyond the built-in scratch: use dps_moe_linear
-    for (int32_t e = 0; e < E; ++e)
-        if (enc_per_expert[e] < DPS_ENC_E4M3 || enc_per_expert[e] > DPS_ENC_E5M2_RN) return DPS_ERR_ENCODING;
-    if (A == 0) return DPS_OK;
-    if (!x || !expert_of_row || !w_persist || !y) return DPS_ERR_NULL;
-    if (mode == DPS_MODE_FULL && !w_resid) return DPS_ERR_NULL;
-    auto misaligned = [](const void* p, uintptr_t mask) { return (reinterpret_cast<uintptr_t>(p) & mask) != 0; };
-    if (misaligned(x, 15) || misaligned(w_persist, 15) || misaligned(y, 15)) return DPS_ERR_ALIGN;
-    if (mode == DPS_MODE_FULL && misaligned(w_resid, 15)) return DPS_ERR_ALIGN;
-    if (misaligned(expert_of_row, 3) || misaligned(token_of_row, 3)) return DPS_ERR_ALIGN;
+    bool empty = false;
+    const dps_status ok = check_moe_args(mode, enc_per_expert, x, token_of_row, expert_of_row, w_persist, w_resid, y, A, T,
+                                         N, K, E, &empty);
+    if (ok != DPS_OK) return ok;
+    if (moe_workspace_bytes(A, E, K) > kStaticScratchBytes) return DPS_ERR_WORKSPACE;  // use dps_moe_linear instead
+    if (empty) return DPS_OK;
     int* status = nullptr;
     const dps_status st = device_status_word(&status);
     if (st != DPS_OK) return st;

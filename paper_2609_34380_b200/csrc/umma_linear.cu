@@ -1242,14 +1242,15 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
     if (stages < 2) stages = 2;
     const size_t smem = (size_t)stages * kStage + kEpiBytes + 1024;
     auto kernel = umma_persistent_kernel<ENC, FULL, TN, GROUPED, RB>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+    static PerDeviceOnce setup;     // per instantiation and per device
+    {
+        const cudaError_t e = setup.run([&] {
+            cudaError_t a = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+            if (a != cudaSuccess) return a;
+            return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        cudaSharedmemCarveoutMaxShared);
+        });
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        configured = true;
     }
     prm.num_stages = stages;
     prm.red_offset = stages * kStage;   // the epilogue's chunk buffer
@@ -1355,48 +1356,58 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     };
     const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kXRing + kMailMax + 1024;
     auto kernel = umma_linear_kernel<ENC, FULL, TN, false>;
-    static int capacity[kMaxSplit + 1] = {0};  // per instantiation; filled on first use
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
-        if (e != cudaSuccess) return e;
-        // Ask for the largest shared-memory carve-out, otherwise the driver may size it for ONE CTA
-        // of this kernel and a second CTA never becomes resident on the SM.
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        for (int s = 1; s <= kMaxSplit; ++s) {
-            cudaLaunchConfig_t q = {};
-            q.gridDim = dim3(1, 1, (unsigned)s);
-            q.blockDim = dim3(kThreads, 1, 1);
-            q.dynamicSmemBytes = smem_query;
-            cudaLaunchAttribute qa[1];
-            qa[0].id = cudaLaunchAttributeClusterDimension;
-            qa[0].val.clusterDim.x = 1;
-            qa[0].val.clusterDim.y = 1;
-            qa[0].val.clusterDim.z = (unsigned)s;
-            q.attrs = qa;
-            q.numAttrs = 1;
-            int clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &q) != cudaSuccess) clusters = 0;
-            capacity[s] = clusters * s;
-        }
-        (void)cudaGetLastError();
-        // The query can be more conservative about CTAs per SM than the hardware turns out to be
-        // (it reported one where two were measured resident); keep its GPC packing ratios and
-        // rescale to the CTAs per SM this kernel is sized for.
-        const int slots = sm_count() * kCtasPerSm;
-        if (capacity[1] <= 0) capacity[1] = slots;
-        const int base = capacity[1];
-        for (int s = 1; s <= kMaxSplit; ++s) capacity[s] = (int)((int64_t)capacity[s] * slots / base);
-        // With two CTAs per SM a cluster of even size s needs only s / 2 SMs of a GPC, so it packs
-        // like a cluster of s / 2 at one CTA per SM (32 row tiles split 8 ways, 256 CTAs, were
-        // measured 5-11 % faster than split 6 ways, which the plain rescaling would have chosen).
-        if (kCtasPerSm == 2)
-            for (int s = kMaxSplit; s >= 2; s -= 2)
-                if (capacity[s / 2] > capacity[s]) capacity[s] = capacity[s / 2];
-        configured = true;
+    // CTAs that can be resident at once for each cluster size: per instantiation and per device, filled by
+    // the first call on that device and read only after that set-up has returned.
+    static int capacity_of[kMaxDevices][kMaxSplit + 1] = {};
+    static PerDeviceOnce setup;
+    int dev = 0;
+    {
+        const cudaError_t e0 = setup.run([&] {
+            int d = 0;
+            cudaGetDevice(&d);
+            int* capacity = capacity_of[d];
+            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+            if (e != cudaSuccess) return e;
+            // Ask for the largest shared-memory carve-out, otherwise the driver may size it for ONE CTA
+            // of this kernel and a second CTA never becomes resident on the SM.
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared);
+            if (e != cudaSuccess) return e;
+            for (int s = 1; s <= kMaxSplit; ++s) {
+                cudaLaunchConfig_t q = {};
+                q.gridDim = dim3(1, 1, (unsigned)s);
+                q.blockDim = dim3(kThreads, 1, 1);
+                q.dynamicSmemBytes = smem_query;
+                cudaLaunchAttribute qa[1];
+                qa[0].id = cudaLaunchAttributeClusterDimension;
+                qa[0].val.clusterDim.x = 1;
+                qa[0].val.clusterDim.y = 1;
+                qa[0].val.clusterDim.z = (unsigned)s;
+                q.attrs = qa;
+                q.numAttrs = 1;
+                int clusters = 0;
+                if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &q) != cudaSuccess) clusters = 0;
+                capacity[s] = clusters * s;
+            }
+            (void)cudaGetLastError();
+            // The query can be more conservative about CTAs per SM than the hardware turns out to be
+            // (it reported one where two were measured resident); keep its GPC packing ratios and
+            // rescale to the CTAs per SM this kernel is sized for.
+            const int slots = sm_count() * kCtasPerSm;
+            if (capacity[1] <= 0) capacity[1] = slots;
+            const int base = capacity[1];
+            for (int s = 1; s <= kMaxSplit; ++s) capacity[s] = (int)((int64_t)capacity[s] * slots / base);
+            // With two CTAs per SM a cluster of even size s needs only s / 2 SMs of a GPC, so it packs
+            // like a cluster of s / 2 at one CTA per SM (32 row tiles split 8 ways, 256 CTAs, were
+            // measured 5-11 % faster than split 6 ways, which the plain rescaling would have chosen).
+            if (kCtasPerSm == 2)
+                for (int s = kMaxSplit; s >= 2; s -= 2)
+                    if (capacity[s / 2] > capacity[s]) capacity[s] = capacity[s / 2];
+            return cudaSuccess;
+        }, &dev);
+        if (e0 != cudaSuccess) return e0;
     }
+    const int* capacity = capacity_of[dev];
     CUtensorMap mp, mr, mx;
     constexpr int kBlockK = block_k(FULL, TN);
     constexpr CUtensorMapSwizzle kPlaneSwizzle = kBlockK == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
@@ -1493,14 +1504,15 @@ cudaError_t launch_tn_rb2(const void* x, const uint8_t* p, const uint8_t* r, voi
     if (stages < 2) stages = 2;
     const size_t smem = (size_t)stages * kStage + 1024;
     auto kernel = umma_linear_kernel<ENC, FULL, TN, false, kRb>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+    static PerDeviceOnce setup;     // per instantiation and per device
+    {
+        const cudaError_t e = setup.run([&] {
+            cudaError_t a = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+            if (a != cudaSuccess) return a;
+            return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        cudaSharedmemCarveoutMaxShared);
+        });
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        configured = true;
     }
     CUtensorMap mp, mr, mx;
     if (!make_map_2d(&mp, p, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, (uint64_t)K, kTileRows * kRb, kBlockK,
@@ -1638,14 +1650,15 @@ cudaError_t launch_grouped_tn(const uint32_t* e5m2_mask, const void* x_sorted, c
     if (stages < 2) stages = 2;
     const size_t smem = (size_t)stages * kStage + 1024;
     auto kernel = umma_linear_kernel<0, FULL, TN, true, RB>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+    static PerDeviceOnce setup;     // per instantiation and per device
+    {
+        const cudaError_t e = setup.run([&] {
+            cudaError_t a = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+            if (a != cudaSuccess) return a;
+            return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                        cudaSharedmemCarveoutMaxShared);
+        });
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        configured = true;
     }
     CUtensorMap mp, mr, mx;
     constexpr int kBlockK = block_k(FULL, TN, RB);

@@ -35,6 +35,17 @@ def assert_close_to_oracle(y_gpu, y_ref: np.ndarray, what=""):
     return err / scale if scale else 0.0
 
 
+def split_both(w: torch.Tensor, enc_req: int, device="cuda:0", p_out=None, r_out=None):
+    """Planes for the GPU (from dps_split_weights) and, independently, the oracle's planes of the same FP16
+    words for the reference side of a parity test: the two paths meet only at their inputs.
+    Returns (p, r, enc, p_ref, r_ref)."""
+    import paper_2609_34380_b200 as dps
+    p, r, enc = dps.dps_split_weights(w.to(device), enc_req, p_out, r_out)
+    p_ref, r_ref, enc_ref = oracle.split(to_np_words(w), enc_req)
+    assert enc == enc_ref, (enc, enc_ref)
+    return p, r, enc, p_ref, r_ref
+
+
 def split_on_host(w: torch.Tensor, enc: int):
     """Oracle split of a (possibly device) FP16 tensor -> numpy planes."""
     return oracle.split(to_np_words(w), enc)

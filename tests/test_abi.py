@@ -96,6 +96,34 @@ def test_host_validation_needs_no_device():
     assert moe(wsb=8) == binding.DPS_ERR_WORKSPACE
     assert moe(ws=odd) == binding.DPS_ERR_WORKSPACE
     assert moe(x=odd) == binding.DPS_ERR_ALIGN
+    # sizes the 32-bit row coordinates of the kernels cannot hold
+    big = 1 << 31
+    assert lib.dps_linear(0, 1, fake, fake, fake, fake, 1, big, 16, None) == binding.DPS_ERR_SHAPE
+    assert lib.dps_linear(0, 1, fake, fake, fake, fake, 1, 8, big, None) == binding.DPS_ERR_SHAPE
+    assert lib.dps_linear(0, 1, fake, fake, fake, fake, big, 8, 16, None) == binding.DPS_ERR_SHAPE
+    assert lib.dps_linear_fp8act(1, fake, fake, fake, fake, 1, big, 16, None) == binding.DPS_ERR_SHAPE
+    many = (ctypes.c_int32 * 1024)(*([1] * 1024))
+    assert moe(enc=many, E=1024, N=1 << 21) == binding.DPS_ERR_SHAPE          # E * N = 2^31
+    assert moe(enc=many, E=1024, N=(1 << 21) - 8, ws=None) == binding.DPS_ERR_WORKSPACE   # just below: accepted so far
+    assert moe(N=big) == binding.DPS_ERR_SHAPE
+    # the allocation-free variant validates the same way (and before it looks for a device)
+    def moe_static(mode=0, enc=encs, x=fake, tor=None, eor=fake, p=fake, r=None, y=fake, **kw):
+        a = {**args, **kw}
+        return lib.dps_moe_linear_static(mode, enc, x, tor, eor, p, r, y, a["A"], a["T"], a["N"], a["K"], a["E"], None)
+    assert moe_static(mode=5) == binding.DPS_ERR_MODE
+    assert moe_static(enc=bad) == binding.DPS_ERR_ENCODING
+    assert moe_static(enc=None) == binding.DPS_ERR_NULL
+    assert moe_static(K=20) == binding.DPS_ERR_SHAPE
+    assert moe_static(E=0) == binding.DPS_ERR_SHAPE
+    assert moe_static(A=0) == binding.DPS_OK
+    assert moe_static(eor=None) == binding.DPS_ERR_NULL
+    assert moe_static(mode=1) == binding.DPS_ERR_NULL
+    assert moe_static(x=odd) == binding.DPS_ERR_ALIGN
+    assert moe_static(enc=many, E=1024, N=1 << 21) == binding.DPS_ERR_SHAPE
+    assert moe_static(A=1 << 20, K=4096) == binding.DPS_ERR_WORKSPACE         # 8 GiB of regrouped activations
+    # diagnostics
+    assert lib.dps_debug_wait_timeout(0, None) == binding.DPS_ERR_SHAPE
+    assert lib.dps_debug_wait_timeout(2_000_000_000, None) == binding.DPS_ERR_SHAPE
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

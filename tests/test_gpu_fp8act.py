@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2609_34380_b200 as dps
 from paper_2609_34380_b200 import workloads
-from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words
+from tests.helpers import assert_close_to_oracle, split_both, to_np_bytes, to_np_words
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -39,11 +39,11 @@ def test_non_finite_activation_raises_the_status_word():
 def test_linear_against_the_oracle(enc_req, N, K, M):
     """Ragged in N (not a multiple of 128), K (partial last block of 128) and M (partial token tile)."""
     w = workloads.weights(N, K, 31, device=DEV)
-    p, r, enc = dps.dps_split_weights(w, enc_req)
+    p, r, enc, p_ref, _ = split_both(w, enc_req, DEV)
     x = workloads.activations(M, K, 32, device=DEV)
     q, scale = dps.dps_quantize_activations(x)
     y = dps.dps_linear_fp8act(enc, q, scale, p)
-    ref = oracle.linear_fp8act(enc, to_np_bytes(q), scale.cpu().numpy(), to_np_bytes(p), threads=8)
+    ref = oracle.linear_fp8act(enc, *oracle.quantize_activations(to_np_words(x)), p_ref, threads=8)   # the oracle's own codes
     assert_close_to_oracle(y, ref, f"fp8act N={N} K={K} M={M} enc={enc}")
     assert torch.equal(y, dps.dps_linear_fp8act(enc, q, scale, p))
     assert dps.dps_stream_status() == dps.DPS_OK
@@ -53,22 +53,22 @@ def test_more_tiles_than_sms_on_256_token_tiles():
     """160 tiles of 128 x 256 on 148 persistent CTAs: both accumulators in use, a second tile for some CTAs."""
     N, K, M = 4096, 272, 1280
     w = workloads.weights(N, K, 33, device=DEV)
-    p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+    p, r, enc, p_ref, _ = split_both(w, dps.DPS_ENC_AUTO, DEV)
     x = workloads.activations(M, K, 34, device=DEV)
     q, scale = dps.dps_quantize_activations(x)
     y = dps.dps_linear_fp8act(enc, q, scale, p)
-    ref = oracle.linear_fp8act(enc, to_np_bytes(q), scale.cpu().numpy(), to_np_bytes(p), threads=16)
+    ref = oracle.linear_fp8act(enc, *oracle.quantize_activations(to_np_words(x)), p_ref, threads=16)   # the oracle's own codes
     assert_close_to_oracle(y, ref, "fp8act 160 tiles")
 
 
 def test_llama_o_proj_512_tokens_and_distance_to_fp16_activations():
     N, K = workloads.LLAMA7B["o"]
     w = workloads.weights(N, K, 2002, device=DEV)
-    p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+    p, r, enc, p_ref, _ = split_both(w, dps.DPS_ENC_AUTO, DEV)
     x = workloads.activations(512, K, 3001, device=DEV)
     q, scale = dps.dps_quantize_activations(x)
     y8 = dps.dps_linear_fp8act(enc, q, scale, p)
-    ref = oracle.linear_fp8act(enc, to_np_bytes(q), scale.cpu().numpy(), to_np_bytes(p), threads=16)
+    ref = oracle.linear_fp8act(enc, *oracle.quantize_activations(to_np_words(x)), p_ref, threads=16)   # the oracle's own codes
     assert_close_to_oracle(y8, ref, "o-proj fp8act")
     y16 = dps.dps_linear(dps.DPS_MODE_FAST, enc, x, p, None)
     diff = (y8.double() - y16.double()).abs().max().item()
@@ -81,14 +81,14 @@ def test_one_hot_activations_pick_out_fast_mode_weights():
     N, K, M = 256, 256, 16
     w = workloads.weights(N, K, 41, device=DEV)
     for enc_req in (dps.DPS_ENC_AUTO, dps.DPS_ENC_E5M2):
-        p, r, enc = dps.dps_split_weights(w, enc_req)
+        p, r, enc, p_ref, _ = split_both(w, enc_req, DEV)
         x = torch.zeros((M, K), dtype=torch.float16, device=DEV)
         ks = [(7 * m + 3) % K for m in range(M)]
         for m, k in enumerate(ks):
             x[m, k] = 1.0
         q, scale = dps.dps_quantize_activations(x)
         y = dps.dps_linear_fp8act(enc, q, scale, p)
-        wf = torch.from_numpy(oracle.fast_words(to_np_bytes(p), enc).view(np.float16).astype(np.float64))
+        wf = torch.from_numpy(oracle.fast_words(p_ref, enc).view(np.float16).astype(np.float64))
         want = torch.stack([wf[:, k] for k in ks]).to(torch.float64)
         # scale = 1/448 in binary32 and q = 448: scale * 448 differs from 1 by at most one binary32 rounding
         assert torch.allclose(y.cpu().double(), want, rtol=2 ** -10, atol=0)

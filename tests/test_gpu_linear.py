@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2609_34380_b200 as dps
 from paper_2609_34380_b200 import workloads
-from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words, y_as_f64
+from tests.helpers import assert_close_to_oracle, split_both, to_np_bytes, to_np_words, y_as_f64
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -15,14 +15,19 @@ ENCS = [dps.DPS_ENC_E4M3, dps.DPS_ENC_E5M2]
 
 
 def planes(n, k, seed, enc, device=DEV):
+    """GPU planes; the oracle's own planes of the same words ride along as p.ref / r.ref."""
     w = workloads.weights(n, k, seed, device=device).to(DEV)
-    p, r, enc = dps.dps_split_weights(w, enc)
-    return w, p, r, enc
+    return (w,) + with_ref(w, enc)
+
+
+def with_ref(w, enc_req):
+    p, r, enc, p.ref, r.ref = split_both(w, enc_req, DEV)
+    return p, r, enc
 
 
 def run_and_check(mode, enc, x, p, r, what):
     y = dps.dps_linear(mode, enc, x, p, r if mode == dps.DPS_MODE_FULL else None)
-    ref = oracle.linear(mode, enc, to_np_words(x), to_np_bytes(p), to_np_bytes(r), threads=8)
+    ref = oracle.linear(mode, enc, to_np_words(x), p.ref, r.ref, threads=8)   # reference side: oracle-made planes
     assert_close_to_oracle(y, ref, what)
     return y
 
@@ -39,7 +44,7 @@ def test_config1(mode, enc):
 @pytest.mark.parametrize("mode", MODES)
 def test_config1_outlier_goes_e5m2(mode):
     w = workloads.with_outlier(workloads.weights(512, 512, 1001)).to(DEV)
-    p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+    p, r, enc = with_ref(w, dps.DPS_ENC_AUTO)
     assert enc == dps.DPS_ENC_E5M2
     x = workloads.activations(4, 512, 1002).to(DEV)
     run_and_check(mode, enc, x, p, r, "cfg1 outlier")
@@ -80,7 +85,7 @@ def test_one_hot_activations_are_bit_exact(M, enc_req):
     full = dps.dps_linear(dps.DPS_MODE_FULL, enc, x, p, r)
     fast = dps.dps_linear(dps.DPS_MODE_FAST, enc, x, p, None)
     w_words = to_np_words(w)
-    fast_words = oracle.fast_words(to_np_bytes(p), enc)
+    fast_words = oracle.fast_words(p.ref, enc)
     # Equality of the FP16 VALUES: for non-zero values that is equality of the bits; a weight
     # that is -0 sums to +0 (0 + (-0) = +0 in IEEE arithmetic, in the oracle as well).
     for m, k in enumerate(ks):
@@ -95,7 +100,7 @@ def test_subnormal_weights_survive():
     w = torch.from_numpy(words.view(np.int16)).view(torch.float16).to(DEV)
     x = torch.full((2, K), 1024.0, dtype=torch.float16, device=DEV)
     for enc_req in ENCS:
-        p, r, enc = dps.dps_split_weights(w, enc_req)
+        p, r, enc = with_ref(w, enc_req)
         for mode in MODES:
             run_and_check(mode, enc, x, p, r, f"subnormal enc={enc} mode={mode}")
 
@@ -136,10 +141,9 @@ def test_llama7b_decode_shapes_sampled():
     oracle recomputes whole output rows for the smallest layer and sampled entries elsewhere."""
     for i, (name, (N, K)) in enumerate(workloads.LLAMA7B.items()):
         w = workloads.weights(N, K, 2001 + i, device=DEV)
-        p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+        p, r, enc, pn, rn = split_both(w, dps.DPS_ENC_AUTO, DEV)
         assert enc == dps.DPS_ENC_E4M3
         del w
-        pn, rn = to_np_bytes(p), to_np_bytes(r)
         for M in workloads.DECODE_M:
             x = workloads.activations(M, K, 2011 + i, device=DEV)
             xn = to_np_words(x)
@@ -157,9 +161,8 @@ def test_llama7b_decode_shapes_sampled():
                 assert np.max(np.abs(got - ref)) <= 2e-3 * scale, (name, M, mode)
         # forced E5M2 on the same shape, M = 8
         w = workloads.weights(N, K, 2001 + i, device=DEV)
-        p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_E5M2)
+        p, r, enc, pn, rn = split_both(w, dps.DPS_ENC_E5M2, DEV)
         del w
-        pn, rn = to_np_bytes(p), to_np_bytes(r)
         x = workloads.activations(8, K, 2011 + i, device=DEV)
         ms, ns = workloads.sample_entries(8, N, 1024, 2998)
         for mode in MODES:

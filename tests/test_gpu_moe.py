@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2609_34380_b200 as dps
 from paper_2609_34380_b200 import workloads
-from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words, y_as_f64
+from tests.helpers import assert_close_to_oracle, split_both, to_np_words, y_as_f64
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -14,14 +14,18 @@ MODES = [dps.DPS_MODE_FAST, dps.DPS_MODE_FULL]
 
 
 def expert_planes(E, N, K, seed, mixed=True):
-    ps, rs, encs = [], [], []
+    """Stacked GPU planes; the oracle's own planes of the same words ride along as p.ref / r.ref, so that
+    the reference side of every comparison is built from the FP16 words, not from the GPU's planes."""
+    ps, rs, encs, p_refs, r_refs = [], [], [], [], []
     for e in range(E):
         w = workloads.weights(N, K, seed + e, device=DEV)
         if mixed and e % 3 == 1:
             w = workloads.with_outlier(w)
-        p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
-        ps.append(p), rs.append(r), encs.append(enc)
-    return torch.stack(ps), torch.stack(rs), encs
+        p, r, enc, p_ref, r_ref = split_both(w, dps.DPS_ENC_AUTO, DEV)
+        ps.append(p), rs.append(r), encs.append(enc), p_refs.append(p_ref), r_refs.append(r_ref)
+    p, r = torch.stack(ps), torch.stack(rs)
+    p.ref, r.ref = np.stack(p_refs), np.stack(r_refs)
+    return p, r, encs
 
 
 @pytest.mark.parametrize("mode", MODES)
@@ -32,7 +36,7 @@ def test_top2_routing_small(mode, E, N, K, T):
     tor, eor = workloads.top2_routing(T, E, 500)
     y = dps.dps_moe_linear(mode, encs, x, torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV), p,
                            r if mode else None)
-    ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r), threads=8)
+    ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, p.ref, r.ref, threads=8)
     assert rc == oracle.OK
     assert_close_to_oracle(y, ref, f"moe E={E}")
     assert dps.dps_stream_status() == dps.DPS_OK
@@ -46,7 +50,7 @@ def test_identity_token_map_and_empty_experts(mode):
     x = workloads.activations(A, K, 700, device=DEV)
     eor = np.random.default_rng(1).choice([0, 2, 5], A).astype(np.int32)     # experts 1, 3, 4 stay empty
     y = dps.dps_moe_linear(mode, encs, x, None, torch.from_numpy(eor).to(DEV), p, r if mode else None)
-    ref, _ = oracle.moe_linear(mode, encs, to_np_words(x), None, eor, to_np_bytes(p), to_np_bytes(r), threads=8)
+    ref, _ = oracle.moe_linear(mode, encs, to_np_words(x), None, eor, p.ref, r.ref, threads=8)
     assert_close_to_oracle(y, ref, "identity map")
 
 
@@ -57,7 +61,7 @@ def test_all_rows_one_expert_equals_dense():
     eor = torch.full((A,), 1, dtype=torch.int32, device=DEV)
     for mode in MODES:
         y = dps.dps_moe_linear(mode, encs, x, None, eor, p, r if mode else None)
-        ref = oracle.linear(mode, encs[1], to_np_words(x), to_np_bytes(p[1]), to_np_bytes(r[1]), threads=8)
+        ref = oracle.linear(mode, encs[1], to_np_words(x), p.ref[1], r.ref[1], threads=8)
         assert_close_to_oracle(y, ref, "one expert")
 
 
@@ -74,7 +78,7 @@ def test_bad_indices_are_skipped_and_flagged():
     dps.dps_moe_linear(dps.DPS_MODE_FULL, encs, x, torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV), p, r, y)
     assert dps.dps_stream_status() == dps.binding.DPS_ERR_DATA
     assert dps.dps_stream_status() == dps.DPS_OK                      # reading clears the word
-    ref, rc = oracle.moe_linear(dps.DPS_MODE_FULL, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r),
+    ref, rc = oracle.moe_linear(dps.DPS_MODE_FULL, encs, to_np_words(x), tor, eor, p.ref, r.ref,
                                 y_init=np.full((2 * T, N), 5.0))
     assert rc == oracle.ERR_DATA
     got = y_as_f64(y)
@@ -97,45 +101,53 @@ def test_fast_mode_ignores_residual_and_is_deterministic():
 
 
 def test_mixtral_shapes_sampled():
-    """Config 4 at full size: 8 experts, hidden 4096, ffn 14336, 256 tokens routed top-2.  The
-    oracle recomputes sampled entries of a few rows per expert."""
+    """Config 4 at full size: 8 experts, hidden 4096, ffn 14336, 256 tokens routed top-2.  Per expert the
+    oracle recomputes eight WHOLE output rows -- the first three, the last three (which sit in the expert's
+    last token tile) and two from the middle of its row list -- and, beyond those, 2048 seeded entries spread
+    over all rows.  The reference planes are the oracle's own split of the FP16 words."""
     E, T = workloads.MIXTRAL_EXPERTS, workloads.MIXTRAL_TOKENS
     tor, eor = workloads.top2_routing(T, E, 4200)
     rng = np.random.default_rng(4999)
     for li, (name, (N, K)) in enumerate(workloads.MIXTRAL_EXPERT.items()):
         p = torch.empty((E, N, K), dtype=torch.uint8, device=DEV)
         r = torch.empty((E, N, K), dtype=torch.uint8, device=DEV)
-        encs = []
+        encs, p_ref, r_ref = [], [], []
         for e in range(E):
             w = workloads.weights(N, K, 4001 + 10 * li + e, device=DEV)
-            _, _, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO, p[e], r[e])
-            encs.append(enc)
+            _, _, enc, pe, re_ = split_both(w, dps.DPS_ENC_AUTO, DEV, p[e], r[e])
+            encs.append(enc), p_ref.append(pe), r_ref.append(re_)
             del w
         if name == "gate_up":
             x = workloads.activations(T, K, 4100, device=DEV)
             tmap = tor
         else:
             x = workloads.activations(2 * T, K, 4300, device=DEV)
-            tmap = None
-        tor_d = None if tmap is None else torch.from_numpy(tmap).to(DEV)
+            tmap = np.arange(2 * T, dtype=np.int32)
+        tor_d = torch.from_numpy(tor).to(DEV) if name == "gate_up" else None
         eor_d = torch.from_numpy(eor).to(DEV)
         xn = to_np_words(x)
-        # rows to check: two rows of every expert
-        rows = np.concatenate([np.nonzero(eor == e)[0][:2] for e in range(E)])
-        cols = rng.integers(0, N, 48)
-        cols[:2] = [0, N - 1]
+        whole = {}
+        for e in range(E):
+            mine = np.nonzero(eor == e)[0]
+            assert len(mine) >= 8
+            mid = mine[len(mine) // 2 - 1:len(mine) // 2 + 1]
+            whole[e] = np.unique(np.concatenate([mine[:3], mid, mine[-3:]]))
+        sa = rng.integers(0, 2 * T, 2048)                   # sampled entries (row a, column n)
+        sn = rng.integers(0, N, 2048)
+        sn[:4] = [0, 1, N - 2, N - 1]
         for mode in MODES:
             y = dps.dps_moe_linear(mode, encs, x, tor_d, eor_d, p, r if mode else None)
             got = y_as_f64(y)
-            for a in rows:
-                e = int(eor[a])
-                t = int(tmap[a]) if tmap is not None else int(a)
-                pe, re_ = to_np_bytes(p[e][cols.tolist()]), to_np_bytes(r[e][cols.tolist()])
-                ref = oracle.linear(mode, encs[e], xn[t:t + 1], pe, re_)[0]
+            for e in range(E):
+                rows = whole[e]
+                ref = oracle.linear(mode, encs[e], xn[tmap[rows]], p_ref[e], r_ref[e], threads=16)
                 scale = np.max(np.abs(ref))
-                assert np.max(np.abs(got[a, cols] - ref)) <= 2e-3 * scale, (name, mode, a)
+                assert np.max(np.abs(got[rows] - ref)) <= 2e-3 * scale, (name, mode, e)
+                sel = np.nonzero(eor[sa] == e)[0]
+                ref_s = oracle.linear_at(mode, encs[e], xn, p_ref[e], r_ref[e], tmap[sa[sel]], sn[sel])
+                assert np.max(np.abs(got[sa[sel], sn[sel]] - ref_s)) <= 2e-3 * np.max(np.abs(ref_s)), (name, mode, e)
         assert dps.dps_stream_status() == dps.DPS_OK
-        del p, r
+        del p, r, p_ref, r_ref
 
 
 @pytest.mark.parametrize("mode", MODES)
@@ -149,7 +161,7 @@ def test_persistent_grouped_kernel_with_short_last_round(mode):
     tor, eor = workloads.top2_routing(T, E, 902)
     args = (mode, encs, x, torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV), p, r if mode else None)
     y = dps.dps_moe_linear(*args)
-    ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r), threads=16)
+    ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, p.ref, r.ref, threads=16)
     assert rc == oracle.OK
     assert_close_to_oracle(y, ref, "grouped persistent")
     assert torch.equal(y, dps.dps_moe_linear(*args))

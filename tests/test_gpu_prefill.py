@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2609_34380_b200 as dps
 from paper_2609_34380_b200 import workloads
-from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words, y_as_f64
+from tests.helpers import assert_close_to_oracle, split_both, to_np_words, y_as_f64
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -17,11 +17,11 @@ def test_o_proj_m512_full_check():
     """O projection, 512 tokens: every output against the FP64 oracle, both modes."""
     N, K = workloads.LLAMA7B["o"]
     w = workloads.weights(N, K, 2002, device=DEV)
-    p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+    p, r, enc, p_ref, r_ref = split_both(w, dps.DPS_ENC_AUTO, DEV)
     x = workloads.activations(512, K, 3001, device=DEV)
     for mode in MODES:
         y = dps.dps_linear(mode, enc, x, p, r if mode else None)
-        ref = oracle.linear(mode, enc, to_np_words(x), to_np_bytes(p), to_np_bytes(r), threads=16)
+        ref = oracle.linear(mode, enc, to_np_words(x), p_ref, r_ref, threads=16)
         assert_close_to_oracle(y, ref, f"o M=512 mode={mode}")
     assert dps.dps_stream_status() == dps.DPS_OK
 
@@ -31,9 +31,8 @@ def test_llama7b_prefill_sampled(M):
     """All four linears at prefill sizes: 16 whole output rows' worth of samples plus random entries."""
     for i, (name, (N, K)) in enumerate(workloads.LLAMA7B.items()):
         w = workloads.weights(N, K, 2001 + i, device=DEV)
-        p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+        p, r, enc, pn, rn = split_both(w, dps.DPS_ENC_AUTO, DEV)
         del w
-        pn, rn = to_np_bytes(p), to_np_bytes(r)
         x = workloads.activations(M, K, 3001 + i, device=DEV)
         xn = to_np_words(x)
         ms, ns = workloads.sample_entries(M, N, 1536, 3999)
@@ -69,11 +68,11 @@ def test_persistent_kernel_ragged_shapes_every_output(enc_req):
     two-row-block tiles; in both the last round is shared out as halves of K.  Every output is checked."""
     N, K, M = 2056, 1104, 2500
     w = workloads.weights(N, K, 611, device=DEV)
-    p, r, enc = dps.dps_split_weights(w, enc_req)
+    p, r, enc, p_ref, r_ref = split_both(w, enc_req, DEV)
     x = workloads.activations(M, K, 612, device=DEV)
     for mode in MODES:
         y = dps.dps_linear(mode, enc, x, p, r if mode else None)
-        ref = oracle.linear(mode, enc, to_np_words(x), to_np_bytes(p), to_np_bytes(r), threads=16)
+        ref = oracle.linear(mode, enc, to_np_words(x), p_ref, r_ref, threads=16)
         assert_close_to_oracle(y, ref, f"ragged persistent mode={mode} enc={enc}")
         again = dps.dps_linear(mode, enc, x, p, r if mode else None)
         assert torch.equal(y, again)              # the pair reduction adds in a fixed order

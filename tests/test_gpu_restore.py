@@ -11,7 +11,7 @@ import torch
 import oracle
 import paper_2609_34380_b200 as dps
 from paper_2609_34380_b200 import workloads
-from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words
+from tests.helpers import assert_close_to_oracle, split_both, to_np_bytes, to_np_words
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -46,7 +46,7 @@ def test_empty_and_argument_checks():
 def test_fast_mode_steps_beside_a_restore_then_full_mode():
     n, k = 4096, 4096
     w = workloads.weights(n, k, 91, device=DEV)
-    p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+    p, r, enc, p_ref, r_ref = split_both(w, dps.DPS_ENC_AUTO, DEV)
     host = dps.dps_backup_residual(r)
     x = workloads.activations(8, k, 92, device=DEV)
     y_alone = dps.dps_linear(dps.DPS_MODE_FAST, enc, x, p, None)
@@ -66,6 +66,7 @@ def test_fast_mode_steps_beside_a_restore_then_full_mode():
     torch.cuda.synchronize()
     for y in ys:
         assert torch.equal(y, y_alone)
-    ref = oracle.linear(oracle.MODE_FULL, enc, to_np_words(x), to_np_bytes(p), host.numpy(), threads=8)
+    assert np.array_equal(host.numpy(), r_ref)
+    ref = oracle.linear(oracle.MODE_FULL, enc, to_np_words(x), p_ref, r_ref, threads=8)
     assert_close_to_oracle(y_full, ref, "full mode after restore")
     assert dps.dps_stream_status() == dps.DPS_OK

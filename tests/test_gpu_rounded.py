@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2609_34380_b200 as dps
 from paper_2609_34380_b200 import workloads
-from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words
+from tests.helpers import assert_close_to_oracle, split_both, to_np_bytes, to_np_words
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -62,10 +62,9 @@ def test_linear_against_the_oracle_in_both_modes(enc, base, N, K, M):
     """Streaming kernel (3, 12 tokens), tcgen05 decode tiles (32), prefill tiles (300) and K halves on CTA
     pairs (200 tokens x 8192 rows); ragged N and K."""
     w = workloads.weights(N, K, 700 + N, device=DEV)
-    p, r, _ = dps.dps_split_weights(w, enc)
+    p, r, _, pn, rn = split_both(w, enc, DEV)        # reference side: the oracle's own planes
     pb, rb, _ = dps.dps_split_weights(w, base)
     x = workloads.activations(M, K, 800 + M, device=DEV)
-    pn, rn = to_np_bytes(p), to_np_bytes(r)
     for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):
         y = dps.dps_linear(mode, enc, x, p, r if mode else None)
         ref = oracle.linear(mode, enc, to_np_words(x), pn, rn, threads=8)
@@ -101,9 +100,9 @@ def test_fp8_activation_fast_mode():
     x = workloads.activations(M, K, 32, device=DEV)
     q, scale = dps.dps_quantize_activations(x)
     for enc, base in PAIRS:
-        p, r, _ = dps.dps_split_weights(w, enc)
+        p, r, _, p_ref, _ = split_both(w, enc, DEV)
         y = dps.dps_linear_fp8act(enc, q, scale, p)
-        ref = oracle.linear_fp8act(enc, to_np_bytes(q), scale.cpu().numpy(), to_np_bytes(p), threads=4)
+        ref = oracle.linear_fp8act(enc, *oracle.quantize_activations(to_np_words(x)), p_ref, threads=4)   # the oracle's own codes
         assert_close_to_oracle(y, ref, f"fp8act rounded enc={enc}")
         assert torch.equal(y, dps.dps_linear_fp8act(base, q, scale, p))
 
@@ -112,20 +111,21 @@ def test_grouped_linear_with_rounded_and_truncated_experts():
     """Experts of all four encodings in one call; one expert with a second token tile, one empty."""
     E, N, K, T = 5, 392, 528, 140
     req = [dps.DPS_ENC_E4M3_RN, dps.DPS_ENC_E5M2, dps.DPS_ENC_E5M2_RN, dps.DPS_ENC_E4M3, dps.DPS_ENC_E4M3_RN]
-    ps, rs, encs = [], [], []
+    ps, rs, encs, p_refs, r_refs = [], [], [], [], []
     for e in range(E):
         w = workloads.weights(N, K, 150 + e, device=DEV)
-        p, r, enc = dps.dps_split_weights(w, req[e])
-        ps.append(p), rs.append(r), encs.append(enc)
+        p, r, enc, p_ref, r_ref = split_both(w, req[e], DEV)
+        ps.append(p), rs.append(r), encs.append(enc), p_refs.append(p_ref), r_refs.append(r_ref)
     assert encs == req
     p, r = torch.stack(ps), torch.stack(rs)
+    p_ref, r_ref = np.stack(p_refs), np.stack(r_refs)
     x = workloads.activations(T, K, 160, device=DEV)
     tor, eor = workloads.top2_routing(T, E, 170)
     eor[eor == E - 1] = 0                         # the last expert stays empty, expert 0 gets two shares
     tor_d, eor_d = torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV)
     for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):
         y = dps.dps_moe_linear(mode, encs, x, tor_d, eor_d, p, r if mode else None)
-        ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r), threads=8)
+        ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, p_ref, r_ref, threads=8)
         assert rc == oracle.OK
         assert_close_to_oracle(y, ref, f"grouped rounded mode={mode}")
         y_static = torch.empty_like(y)

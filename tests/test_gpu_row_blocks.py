@@ -15,12 +15,13 @@ REPO = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _cases():
+    import numpy as np
     import torch
 
     import oracle
     import paper_2609_34380_b200 as dps
     from paper_2609_34380_b200 import workloads
-    from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words
+    from tests.helpers import assert_close_to_oracle, split_both, to_np_words
 
     dev = "cuda:0"
     # dense: N not a multiple of 256 (second row block ragged or absent), K with a ragged last block,
@@ -28,31 +29,31 @@ def _cases():
     for (N, K, M) in [(640, 1088, 200), (128, 512, 65), (904, 2064, 300), (392, 272, 577)]:
         for forced_enc in (dps.DPS_ENC_AUTO, dps.DPS_ENC_E5M2):
             w = workloads.weights(N, K, 11 + N, device=dev)
-            p, r, enc = dps.dps_split_weights(w, forced_enc)
+            p, r, enc, p_ref, r_ref = split_both(w, forced_enc, dev)
             x = workloads.activations(M, K, 13 + M, device=dev)
             for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):
                 y = dps.dps_linear(mode, enc, x, p, r if mode else None)
-                ref = oracle.linear(mode, enc, to_np_words(x), to_np_bytes(p), to_np_bytes(r), threads=8)
+                ref = oracle.linear(mode, enc, to_np_words(x), p_ref, r_ref, threads=8)
                 assert_close_to_oracle(y, ref, f"dense N={N} K={K} M={M} enc={enc} mode={mode}")
                 print(f"ok dense N={N} K={K} M={M} enc={enc} mode={mode}")
     # grouped: experts with 0, few and more than one tile of rows; N ragged against 256
     for (E, N, K, T) in [(4, 384, 1040, 90), (3, 136, 528, 150)]:
-        ps, rs, encs = [], [], []
+        ps, rs, encs, p_refs, r_refs = [], [], [], [], []
         for e in range(E):
             w = workloads.weights(N, K, 50 + e, device=dev)
             if e == 1:
                 w = workloads.with_outlier(w)
-            p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
-            ps.append(p), rs.append(r), encs.append(enc)
+            p, r, enc, p_ref, r_ref = split_both(w, dps.DPS_ENC_AUTO, dev)
+            ps.append(p), rs.append(r), encs.append(enc), p_refs.append(p_ref), r_refs.append(r_ref)
         p, r = torch.stack(ps), torch.stack(rs)
+        p_ref, r_ref = np.stack(p_refs), np.stack(r_refs)
         x = workloads.activations(T, K, 60, device=dev)
         tor, eor = workloads.top2_routing(T, E, 70)
         eor[eor == E - 1] = 0                     # the last expert stays empty, expert 0 gets two shares
         for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):
             y = dps.dps_moe_linear(mode, encs, x, torch.from_numpy(tor).to(dev), torch.from_numpy(eor).to(dev), p,
                                    r if mode else None)
-            ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, to_np_bytes(p), to_np_bytes(r),
-                                        threads=8)
+            ref, rc = oracle.moe_linear(mode, encs, to_np_words(x), tor, eor, p_ref, r_ref, threads=8)
             assert rc == oracle.OK
             assert_close_to_oracle(y, ref, f"grouped E={E} N={N} mode={mode}")
             print(f"ok grouped E={E} N={N} K={K} T={T} mode={mode}")

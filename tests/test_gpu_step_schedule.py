@@ -7,7 +7,7 @@ import torch
 import oracle
 import paper_2609_34380_b200 as dps
 from paper_2609_34380_b200 import workloads
-from tests.helpers import assert_close_to_oracle, to_np_bytes, to_np_words, y_as_f64
+from tests.helpers import assert_close_to_oracle, split_both, to_np_words, y_as_f64
 
 gpu = pytest.mark.gpu
 DEV = "cuda:0"
@@ -18,13 +18,15 @@ class MiniDecoder:
 
     def __init__(self, layers, shapes, M, seed):
         self.shapes, self.M = shapes, M
-        self.planes = []
+        self.planes, self.ref_planes = [], []              # GPU planes; the oracle's own planes of the same words
         for layer in range(layers):
-            row = {}
+            row, ref_row = {}, {}
             for i, (name, (n, k)) in enumerate(shapes.items()):
                 w = workloads.weights(n, k, seed + layer * 4 + i, device=DEV)
-                row[name] = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+                p, r, enc, p_ref, r_ref = split_both(w, dps.DPS_ENC_AUTO, DEV)
+                row[name], ref_row[name] = (p, r, enc), (p_ref, r_ref)
             self.planes.append(row)
+            self.ref_planes.append(ref_row)
         self.x = {name: workloads.activations(M, k, 5901 + i, device=DEV) for i, (name, (n, k)) in enumerate(shapes.items())}
         self.y = {(layer, name): torch.zeros((M, n), dtype=torch.float16, device=DEV)
                   for layer in range(layers) for name, (n, k) in shapes.items()}
@@ -78,7 +80,8 @@ def test_schedule_outputs_depend_only_on_the_mode_of_the_step(M):
     # layer 0 against the oracle, both modes
     for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):
         for name, (p, r, enc) in model.planes[0].items():
-            ref = oracle.linear(mode, enc, to_np_words(model.x[name]), to_np_bytes(p), to_np_bytes(r), threads=16)
+            p_ref, r_ref = model.ref_planes[0][name]
+            ref = oracle.linear(mode, enc, to_np_words(model.x[name]), p_ref, r_ref, threads=16)
             assert_close_to_oracle(first[mode][(0, name)], ref, f"{name} mode={mode}")
     assert dps.dps_stream_status() == dps.DPS_OK
 
@@ -99,13 +102,13 @@ def test_decoder70_layer_shapes_sampled(M):
     """Config 5 shapes (hidden 8192, ffn 28672, GQA QKV): one layer at full size, sampled outputs."""
     for i, (name, (N, K)) in enumerate(workloads.DECODER70.items()):
         w = workloads.weights(N, K, 5000 + i, device=DEV)
-        p, r, enc = dps.dps_split_weights(w, dps.DPS_ENC_AUTO)
+        p, r, enc, p_ref, r_ref = split_both(w, dps.DPS_ENC_AUTO, DEV)
         del w
         x = workloads.activations(M, K, 5901 + i, device=DEV)
         ms, ns = workloads.sample_entries(M, N, 768, 5999 + M)
         ns[:4] = [0, 127, 128, N - 1]
         rows = np.unique(ns)
-        pn, rn = to_np_bytes(p[rows.tolist()]), to_np_bytes(r[rows.tolist()])
+        pn, rn = p_ref[rows], r_ref[rows]                  # reference side: the oracle's own planes
         idx = np.searchsorted(rows, ns)
         xn = to_np_words(x)
         for mode in (dps.DPS_MODE_FAST, dps.DPS_MODE_FULL):

@@ -9,7 +9,6 @@ Who needs this entry point: callers that are not allowed to allocate device memo
 run -- for instance a serving worker that committed all free memory to weight planes and KV
 cache at start-up -- and therefore cannot provide the workspace dps_moe_linear asks for.
 """
-import numpy as np
 import pytest
 import torch
 
@@ -18,7 +17,6 @@ from paper_2609_34380_b200 import binding, workloads
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
-REL_BOUND = 2e-3      # the tight bound the other GEMM parity tests use
 
 
 def _problem(E, N, K, T, seed):
@@ -40,9 +38,9 @@ def _compare(mode, prob):
     got = torch.full_like(want, 7.0)
     dps.dps_moe_linear_static(mode, encs, x, tor, eor, p, r if mode else None, got)
     torch.cuda.synchronize()
-    a, b = got.double().cpu().numpy(), want.double().cpu().numpy()
-    assert np.all(np.isfinite(a))
-    assert np.max(np.abs(a - b)) <= REL_BOUND * np.max(np.abs(b))
+    # the two entry points run the same deterministic kernels: the outputs must agree bit for bit
+    assert bool(torch.isfinite(got).all())
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
     return got
 
 
