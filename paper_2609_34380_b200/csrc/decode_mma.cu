@@ -47,6 +47,21 @@ __device__ __forceinline__ uint4 ldg_stream(const void* p) {
     return v;
 }
 
+// Optional timeline (compile with -DDPS_TRACE): time stamps of the CTAs of the last eight launches, read
+// back with dps_debug_decode_times().
+#ifdef DPS_TRACE
+constexpr int kTraceCtas = 1536, kTraceEvents = 8, kTraceLaunches = 8;
+__device__ unsigned long long g_decode_times[kTraceLaunches * kTraceCtas * kTraceEvents];
+#define DPS_DSTAMP(ev)                                                                                          \
+    do {                                                                                                        \
+        if (threadIdx.x == 0 && blockIdx.x < kTraceCtas)                                                        \
+            g_decode_times[((trace_slot % kTraceLaunches) * kTraceCtas + blockIdx.x) * kTraceEvents + (ev)] =  \
+                sm100::global_timer_ns();                                                                       \
+    } while (0)
+#else
+#define DPS_DSTAMP(ev) do { } while (0)
+#endif
+
 // D (16x8, FP32) += A (16x16 FP16, row) * B (16x8 FP16, col)
 __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                           uint32_t b0, uint32_t b1) {
@@ -73,10 +88,11 @@ template <int ENC, bool FULL, int NT, int U, bool HALF>
 __global__ void __launch_bounds__(kThreads, (FULL && NT == 1 && U == 2) ? 3 : 2)
 decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, const uint8_t* __restrict__ Rp,
                   __half* __restrict__ y, int M, int64_t N, int64_t K, int prefetch_steps,
-                  int prefetch_ctas) {
+                  int prefetch_ctas, int trace_slot) {
     constexpr float kScale = (ENC == kEncE4M3 && !FULL) ? 0.00390625f : 1.0f;  // 2^-8, exact
     __shared__ float red[kWarps][kRowsPerBlock][NT * 8 + 1];
     sm100::grid_launch_dependents();
+    DPS_DSTAMP(0);
     // A CTA that becomes resident while the preceding kernel drains has no activations yet (they are
     // that kernel's output), but its weights are model state: the first batch of weight loads is
     // issued BEFORE the dependency wait (below), and the first wave of CTAs asks L2 for the stretch
@@ -172,7 +188,11 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
             }
             // Everything but the planes may come from the preceding kernel: wait for it here, with the
             // first batch of weight loads already in flight.
-            if (r0 == 0) sm100::grid_dependency_wait();
+            if (r0 == 0) {
+                DPS_DSTAMP(1);
+                sm100::grid_dependency_wait();
+                DPS_DSTAMP(2);
+            }
             // the activation fragments of the batch are fetched together with the weights, so that
             // their (L1 / L2) latency hides behind the DRAM latency of the weight loads
             uint4 xb[U][NT][2];
@@ -213,6 +233,10 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
             }
         }
         // accumulator fragment: c0,c1 = (row g, tokens 2t, 2t+1), c2,c3 = (row g+8, same tokens)
+#ifdef DPS_TRACE
+        asm volatile("" ::"f"(acc[0][0] + acc[0][3]));
+        DPS_DSTAMP(3);
+#endif
 #pragma unroll
         for (int n = 0; n < NT; ++n) {
             red[warp][g][n * 8 + 2 * t] = acc[n][0];
@@ -234,6 +258,7 @@ decode_mma_kernel(const __half* __restrict__ x, const uint8_t* __restrict__ P, c
             }
         }
         __syncthreads();
+        DPS_DSTAMP(4);
     }
 }
 
@@ -264,8 +289,13 @@ cudaError_t launch_one(const __half* x, const uint8_t* p, const uint8_t* r, __ha
         const char* e = getenv("DPS_STREAM_PREFETCH_CTAS");
         return e ? atoi(e) : 2 * sm_count();
     }();
+    int trace_slot = 0;
+#ifdef DPS_TRACE
+    static int trace_launches = 0;
+    trace_slot = trace_launches++;
+#endif
     cudaError_t e = cudaLaunchKernelEx(&cfg, decode_mma_kernel<ENC, FULL, NT, U, HALF>, x, p, r, y, M, N, K,
-                                       prefetch_steps, prefetch_ctas);
+                                       prefetch_steps, prefetch_ctas, trace_slot);
     count_launch();
     return e;
 }
@@ -311,5 +341,11 @@ cudaError_t launch_decode_mma(int mode, int enc, const void* x, const uint8_t* p
     return full ? launch_enc<kEncE5M2, true>(xh, p, r, yh, (int)M, N, K, stream)
                 : launch_enc<kEncE5M2, false>(xh, p, r, yh, (int)M, N, K, stream);
 }
+
+#ifdef DPS_TRACE
+extern "C" __attribute__((visibility("default"))) int dps_debug_decode_times(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, g_decode_times, sizeof(g_decode_times));
+}
+#endif
 
 }  // namespace dps
