@@ -113,7 +113,10 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
 #ifndef DPS_XSLOT_MAX_TN
 #define DPS_XSLOT_MAX_TN 32
 #endif
-constexpr int kMaxXSlots = 3;
+#ifndef DPS_XSLOTS
+#define DPS_XSLOTS 3
+#endif
+constexpr int kMaxXSlots = DPS_XSLOTS;
 __host__ __device__ constexpr int x_slots(bool grouped, int tn, int rb) {
     return (!grouped && rb == 1 && tn >= DPS_XSLOT_MIN_TN && tn <= DPS_XSLOT_MAX_TN) ? kMaxXSlots : 0;
 }
@@ -211,7 +214,8 @@ struct ZipState {
 // (Measured and dropped for single-row-block 256-token tiles: both groups rebuilding half of every K
 // block -- half the time from a stage's arrival to its A slot being ready, same throughput -- was
 // 4 % slower than alternating blocks.)
-template <int ENC, bool FULL, int TN, int RB>
+// EARLY: the stage holds planes only, so it is handed back as soon as this warp has it in registers.
+template <int ENC, bool FULL, int TN, int RB, bool EARLY = false>
 __device__ __forceinline__ bool zip_blocks(const ZipCtx& z, ZipState& st) {
     constexpr int kBlockK = block_k(FULL, TN, RB);
     constexpr int kACols = kBlockK / 2;
@@ -261,6 +265,10 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z, ZipState& st) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) h[c * 8 + j] = h8[j];
         }
+        if (EARLY) {
+            __syncwarp();
+            if (z.lane == 0) mbar_arrive(smem_u32(&z.bar_empty[s]));
+        }
         ok = mbar_wait(smem_u32(&z.bar_a_empty[a]), a_parity ^ 1u);   // now the slot must be free
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
@@ -279,7 +287,7 @@ __device__ __forceinline__ bool zip_blocks(const ZipCtx& z, ZipState& st) {
         __syncwarp();
         if (z.lane == 0) {
             mbar_arrive(smem_u32(&z.bar_a_full[a]));
-            mbar_arrive(smem_u32(&z.bar_empty[s]));
+            if (!EARLY) mbar_arrive(smem_u32(&z.bar_empty[s]));
         }
         if (z.warp == 2 + 4 * z.group) DPS_STAMP(8, i);
     }
@@ -317,6 +325,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     __shared__ __align__(8) uint64_t bar_a_empty[kMaxAStages];
     __shared__ __align__(8) uint64_t bar_d_full;
     __shared__ __align__(8) uint64_t bar_x_full[kMaxXSlots];
+    __shared__ __align__(8) uint64_t bar_x_empty[kMaxXSlots];
+    __shared__ __align__(8) uint64_t bar_dep;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int s_rows[GROUPED ? TN : 1];   // grouped launches: row ids of the tile's tokens
 
@@ -381,14 +391,20 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     if (threadIdx.x == 0) {
         for (int s = 0; s < num_stages; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_empty[s]), RB == 2 ? 9 : 5);  // 4 zip warps per reader group + 1 tcgen05.commit
+            // 4 zip warps per reader group + 1 tcgen05.commit; a stage that holds planes only (the activations
+            // have slots) is read by the zip warps alone
+            mbar_init(smem_u32(&bar_empty[s]), RB == 2 ? 9 : (kXS ? 4 : 5));
         }
         for (int a = 0; a < kMaxAStages; ++a) {
             mbar_init(smem_u32(&bar_a_full[a]), 4);
             mbar_init(smem_u32(&bar_a_empty[a]), 1);
         }
         mbar_init(smem_u32(&bar_d_full), 1);
-        for (int a = 0; a < kMaxXSlots; ++a) mbar_init(smem_u32(&bar_x_full[a]), 1);
+        for (int a = 0; a < kMaxXSlots; ++a) {
+            mbar_init(smem_u32(&bar_x_full[a]), 1);
+            mbar_init(smem_u32(&bar_x_empty[a]), 1);   // the tcgen05.commit behind the MMAs that read the slot
+        }
+        mbar_init(smem_u32(&bar_dep), 1);
         fence_barrier_init();
         prefetch_tensormap(&map_p);
         if (FULL) prefetch_tensormap(&map_r);
@@ -461,33 +477,23 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         }
         __syncwarp();
         DPS_CTA_STAMP_T(8, 0);
-        if (!GROUPED) grid_dependency_wait();   // grouped launches waited before reading the tile list
-        DPS_CTA_STAMP_T(9, 0);
-        if (elect_one()) {
-            if (kXS) {
-                for (int j = 0; j < kXS && j < num_kb; ++j) load_x_slot(j, j);
-            } else {
-                for (int i = 0; i < first; ++i) {
-                    if (GROUPED) load_planes(i, i);
-                    load_x(i, i);
-                }
+        // grouped launches waited before reading the tile list; with activation slots the MMA warp waits and
+        // reports on bar_dep, so that this warp can go on requesting planes meanwhile
+        if (!GROUPED && !kXS) grid_dependency_wait();
+        if (!kXS) DPS_CTA_STAMP_T(9, 0);
+        if (!kXS && elect_one()) {
+            for (int i = 0; i < first; ++i) {
+                if (GROUPED) load_planes(i, i);
+                load_x(i, i);
             }
         }
         __syncwarp();
-        // Steady state.  Without activation slots: wait for stage s to be free, refill it (planes
-        // and activations of K block i).  With slots: the activations of block i - lag, lag =
-        // depth - slots, are requested in the same step as the planes of block i.  Their slot was
-        // last read by the MMA of block i - depth, the very MMA whose completion freed stage s, so
-        // the one wait covers both; the loop runs `lag` steps past the last plane load to request
-        // the remaining activation tiles.
-        const int lag = kXS ? num_stages - kXS : 0;
-        const int begin = kXS ? num_stages : first;
-        int s = begin == num_stages ? 0 : begin;
-        uint32_t ph = begin == num_stages ? 1u : 0u;
-        int xslot = 0;   // slot of block i - lag: the first such block is block kXS, i.e. slot 0 again
-        const int extra = lag > 0 ? lag : 0;   // a ring shallower than the slots makes the lag negative: nothing to add
-        for (int i = begin; i < num_kb + extra && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
-            if (!pair || (i & 1) == 0 || i >= num_kb) {
+        // Steady state without activation slots: wait for stage s to be free, refill it (planes and
+        // activations of K block i).
+        int s = first == num_stages ? 0 : first;
+        uint32_t ph = first == num_stages ? 1u : 0u;
+        for (int i = first; !kXS && i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, ph ^= (s == 0)) {
+            if (!pair || (i & 1) == 0) {
                 ok = mbar_wait(smem_u32(&bar_empty[s]), ph ^ 1u);
                 if (ok && pair && (i & 1) == 0 && i + 1 < num_kb) {     // pairs never wrap: the ring depth is even
                     ok = mbar_wait(smem_u32(&bar_empty[s + 1]), ph ^ 1u);
@@ -497,28 +503,70 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             if (!ok) break;
             DPS_STAMP(0, i);
             if (elect_one()) {
-                if (i < num_kb) load_planes(i, s);
-                if (kXS) {
-                    if (i - lag < num_kb) load_x_slot(i - lag, xslot);
-                    xslot = (xslot + 1 == kXS) ? 0 : xslot + 1;
-                } else {
-                    load_x(i, s);
-                }
+                load_planes(i, s);
+                load_x(i, s);
             }
             __syncwarp();
+        }
+        // Steady state with activation slots: two streams with different consumers.  A plane stage is free as
+        // soon as its zip group holds it in registers; an activation slot is free when the MMAs that read it
+        // are complete, several K blocks later.  One loop serves both by PROBING (test_wait never suspends)
+        // whichever barrier comes next in each stream, so that neither stream waits for the other's consumer;
+        // the clock is read once in a while to keep the wait bounded.
+        if (kXS) {
+            int ip = first, ix = 0;                                     // next K block of each stream
+            int sp = first == num_stages ? 0 : first, sx = 0;           // its stage / slot
+            uint32_t php = 0u, phx = 0u;                                // parity of the "free" phase awaited there
+            bool dep = false;                                           // the preceding kernel's output may be read
+            uint32_t idle = 0;
+            unsigned long long t0 = 0;
+            while ((ip < num_kb || ix < num_kb) && ok) {
+                bool progress = false;
+                if (ip < num_kb && __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_empty[sp]), php))) {
+                    DPS_STAMP(0, ip);
+                    if (elect_one()) load_planes(ip, sp);
+                    __syncwarp();
+                    ++ip;
+                    sp = (sp + 1 == num_stages) ? 0 : sp + 1;
+                    php ^= (sp == 0);
+                    progress = true;
+                }
+                if (!dep && __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_dep), 0u))) {
+                    grid_dependency_wait();     // returns at once; orders this warp's loads behind the dependency
+                    DPS_CTA_STAMP_T(9, 0);
+                    dep = true;
+                }
+                if (dep && ix < num_kb &&
+                    (ix < kXS || __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_x_empty[sx]), phx)))) {
+                    if (elect_one()) load_x_slot(ix, sx);
+                    __syncwarp();
+                    ++ix;
+                    sx = (sx + 1 == kXS) ? 0 : sx + 1;
+                    if (sx == 0 && ix > kXS) phx ^= 1u;
+                    progress = true;
+                }
+                if (progress) {
+                    idle = 0;
+                } else if ((++idle & 1023u) == 0) {
+                    const unsigned long long now = global_timer_ns();
+                    if (idle == 1024u) t0 = now;
+                    else if (now - t0 > kWaitLimitNs) ok = false;
+                }
+            }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (whole warp converged, one elected lane issues) ----------------
         constexpr int kTotalSlots = a_slots_max(FULL, TN);
-        int s = 0;
-        uint32_t s_parity = 0;
-        int cnt[2] = {0, 0};     // K blocks taken from each zip group so far
-        int xslot = 0;           // activation slot of K block i (tiles with activation slots)
-        uint32_t xparity = 0;
-        for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1, s_parity ^= (s == 0)) {
-            const uint32_t xbase = kXS ? smem_base + (uint32_t)prm.x_offset + (uint32_t)(xslot * kXBytes)
-                                       : smem_base + (uint32_t)s * kStage + kXOffset;
-            if (RB == 2) {
+        if (kXS) {
+            // idle until the first activations arrive anyway: waits for the preceding kernel on the producer's behalf
+            grid_dependency_wait();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_dep));
+            __syncwarp();
+        }
+        if constexpr (RB == 2) {
+            int s = 0;
+            for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1) {
+                const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
                 // row block g: A slot 2g + (i & 1) of zip group g, accumulator columns [g * TN, (g + 1) * TN)
 #pragma unroll
                 for (int g = 0; g < 2; ++g) {
@@ -546,45 +594,89 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                     __syncwarp();
                 }
                 DPS_STAMP(3, i);
-                continue;
             }
-            // stage s belongs to zip group s % 2, which rotates through its own A slots (see zip_blocks)
-            const int g = s & 1;
-            const int g_slots = (kTotalSlots - g + 1) / 2;             // 1 or 2
-            const int turn = g_slots == 2 ? (cnt[g] & 1) : 0;
-            const int a = g + 2 * turn;
-            const uint32_t a_parity = (uint32_t)(g_slots == 2 ? (cnt[g] >> 1) : cnt[g]) & 1u;
-            ++cnt[g];
-            // The zip warps waited for this stage's TMA loads before they arrived on a_full, so the
-            // activation tile of the stage is complete and visible once a_full is: one wait, not two.
-            DPS_STAMP(1, i);
-            ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
-            // ... unless the activations have slots of their own: then their barrier is waited for too
-            if (kXS && ok) ok = mbar_wait(smem_u32(&bar_x_full[xslot]), xparity);
-            if (kXS) {
-                xslot = (xslot + 1 == kXS) ? 0 : xslot + 1;
-                xparity ^= (xslot == 0);
-            }
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            DPS_STAMP(2, i);
-            if (i == 0) DPS_CTA_STAMP_T(10, 32);
-            tc_fence_after_sync();
-            if (elect_one()) {
-#pragma unroll
-                for (int j = 0; j < kBlockK / 16; ++j) {
-                    // 16 K elements = 32 bytes inside the 128-byte swizzle atom (j / 4)
-                    const uint64_t bdesc = umma_desc_k_sw128(xbase + (uint32_t)((j >> 2) * TN * 128)) +
-                                           (uint64_t)((j & 3) * 2);
-                    umma_f16_ts(tmem_d, tmem_a + (uint32_t)(a * kACols + j * 8), bdesc, idesc,
-                                (i > 0 || j > 0) ? 1u : 0u);
+        } else {
+            // Stage s belongs to zip group s % 2, which rotates through its own A slots (see zip_blocks); the
+            // activation tile rides in the stage or sits in slot i % kXS.  The zip warps waited for the stage's
+            // TMA loads before they arrived on a_full, so a tile inside the stage is complete once a_full is;
+            // a tile in a slot has a barrier of its own.
+            //
+            // With 32-token tiles a K block is 4 or 8 short MMAs, and a wait, an MMA batch and the commits each
+            // cost this warp 150-200 cycles of latency (850-900 cycles per K block were measured when they ran
+            // one after the other, more than the planes take to arrive).  So the barriers of block i + 1 are
+            // PROBED (test_wait, which never suspends) before the MMAs of block i are issued, and only a block
+            // that was not ready by then is waited for.
+            int s = 0, xslot = 0;
+            uint32_t xparity = 0, cnt0 = 0, cnt1 = 0;   // K blocks taken from each zip group so far
+            auto a_slot_of = [&](int stage, uint32_t& a_parity) -> int {
+                constexpr int g0_slots = (kTotalSlots + 1) / 2, g1_slots = kTotalSlots / 2;   // 1 or 2 each
+                if ((stage & 1) == 0) {
+                    a_parity = (g0_slots == 2 ? cnt0 >> 1 : cnt0) & 1u;
+                    return g0_slots == 2 ? 2 * (int)(cnt0 & 1u) : 0;
                 }
-                umma_commit(smem_u32(&bar_empty[s]));
-                umma_commit(smem_u32(&bar_a_empty[a]));
-                if (i == num_kb - 1) umma_commit(smem_u32(&bar_d_full));
+                a_parity = (g1_slots == 2 ? cnt1 >> 1 : cnt1) & 1u;
+                return g1_slots == 2 ? 1 + 2 * (int)(cnt1 & 1u) : 1;
+            };
+            uint32_t a_parity = 0;
+            int a = a_slot_of(0, a_parity);
+            DPS_STAMP(1, 0);
+            if (num_kb > 0) {
+                ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
+                DPS_CTA_STAMP_T(11, 32);
+                if (kXS && ok) ok = mbar_wait(smem_u32(&bar_x_full[0]), 0u);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                DPS_CTA_STAMP_T(10, 32);
             }
-            __syncwarp();
-            DPS_STAMP(3, i);
+            for (int i = 0; i < num_kb && ok; ++i) {
+                DPS_STAMP(2, i);
+                const uint32_t xbase = kXS ? smem_base + (uint32_t)prm.x_offset + (uint32_t)(xslot * kXBytes)
+                                           : smem_base + (uint32_t)s * kStage + kXOffset;
+                // block i is taken: advance the group's count, then look at block i + 1
+                if ((s & 1) == 0) ++cnt0; else ++cnt1;
+                const int s1 = (s + 1 == num_stages) ? 0 : s + 1;
+                int xslot1 = xslot;
+                uint32_t xparity1 = xparity;
+                if (kXS) {
+                    xslot1 = (xslot + 1 == kXS) ? 0 : xslot + 1;
+                    xparity1 ^= (xslot1 == 0);
+                }
+                uint32_t a1_parity = 0;
+                const int a1 = a_slot_of(s1, a1_parity);
+                bool next_ready = false;
+                if (i + 1 < num_kb) {
+                    next_ready = mbar_test_wait(smem_u32(&bar_a_full[a1]), a1_parity);
+                    if (kXS) next_ready = mbar_test_wait(smem_u32(&bar_x_full[xslot1]), xparity1) && next_ready;
+                }
+                tc_fence_after_sync();
+                if (elect_one()) {
+#pragma unroll
+                    for (int j = 0; j < kBlockK / 16; ++j) {
+                        // 16 K elements = 32 bytes inside the 128-byte swizzle atom (j / 4)
+                        const uint64_t bdesc = umma_desc_k_sw128(xbase + (uint32_t)((j >> 2) * TN * 128)) +
+                                               (uint64_t)((j & 3) * 2);
+                        umma_f16_ts(tmem_d, tmem_a + (uint32_t)(a * kACols + j * 8), bdesc, idesc,
+                                    (i > 0 || j > 0) ? 1u : 0u);
+                    }
+                    DPS_STAMP(10, i);
+                    if (kXS) umma_commit(smem_u32(&bar_x_empty[xslot]));   // the slot may be refilled ...
+                    else umma_commit(smem_u32(&bar_empty[s]));             // ... or the stage that holds the tile
+                    umma_commit(smem_u32(&bar_a_empty[a]));
+                    if (i == num_kb - 1) umma_commit(smem_u32(&bar_d_full));
+                }
+                __syncwarp();
+                DPS_STAMP(3, i);
+                if (i + 1 < num_kb) {
+                    next_ready = __all_sync(0xFFFFFFFFu, next_ready);
+                    if (!next_ready) {
+                        DPS_STAMP(1, i + 1);
+                        ok = mbar_wait(smem_u32(&bar_a_full[a1]), a1_parity);
+                        DPS_STAMP(9, i + 1);
+                        if (kXS && ok) ok = mbar_wait(smem_u32(&bar_x_full[xslot1]), xparity1);
+                        ok = __all_sync(0xFFFFFFFFu, ok);
+                    }
+                }
+                s = s1; a = a1; xslot = xslot1; xparity = xparity1;
+            }
         }
     } else {
         // ---------------- zip warps: planes -> FP16 -> tensor memory; then epilogue ----------------
@@ -612,7 +704,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
         } else {
             ZipState zst;
-            ok = zip_blocks<ENC, FULL, TN, RB>(zc, zst);
+            ok = zip_blocks<ENC, FULL, TN, RB, (kXS > 0)>(zc, zst);
         }
         // E4M3 fast mode multiplied with 2^8 times the weights (hardware FP8 conversion)
         const float out_scale = (!FULL && !e5m2) ? 0.00390625f : 1.0f;
