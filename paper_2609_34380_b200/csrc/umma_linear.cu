@@ -98,15 +98,15 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
     return c;
 }
 
-// Activation slots kept apart from the plane ring.  Decode tiles (dense launches, 32 tokens):
-// the activation tile is a third to a fifth of a stage, yet it is needed only when the MMA runs,
-// a DRAM latency after the planes were requested.  Three slots of their own, filled three K blocks
-// ahead of the MMA out of L2, let the same shared memory hold one more plane stage in flight.
-// (Two slots were measured: under load the L2 fetch takes longer than two K blocks, and the MMA
-// warp waited for activations.)  0 = the activation tile travels inside the stage.
-// Not for 64-token tiles: their activation tile is as large as a plane stage, and three slots
-// would leave a ring of two.  Not for 16-token tiles either: measured 2-6 % slower there (the
-// tile is a fifth of a stage, so the slots buy no extra stage).
+// Activation slots kept apart from the plane ring.  Decode tiles (dense launches, 32 tokens): the plane
+// stage and the activation tile of a K block have different consumers -- the zip warps take the planes into
+// registers and hand the stage back at once, the MMAs read the activations several K blocks later -- and a
+// tile fetched by the copy engine was measured to arrive 2000-2400 cycles after its request even out of L2.
+// So the tiles get slots of their own, requested as soon as the MMAs that read a slot last are complete,
+// five K blocks ahead (three were 2-4 % slower on most Llama-7B shapes in both modes, six and eight leave
+// too few plane stages in fast mode).  0 = the activation tile travels inside the stage.
+// Not for 64-token tiles: their activation tile is as large as a plane stage, and the slots would leave a
+// ring of two.  Not for 16-token tiles either: measured 2-6 % slower there.
 #ifndef DPS_XSLOT_MIN_TN
 #define DPS_XSLOT_MIN_TN 32
 #endif
@@ -114,7 +114,7 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
 #define DPS_XSLOT_MAX_TN 32
 #endif
 #ifndef DPS_XSLOTS
-#define DPS_XSLOTS 3
+#define DPS_XSLOTS 5
 #endif
 constexpr int kMaxXSlots = DPS_XSLOTS;
 __host__ __device__ constexpr int x_slots(bool grouped, int tn, int rb) {
@@ -600,53 +600,32 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             // activation tile rides in the stage or sits in slot i % kXS.  The zip warps waited for the stage's
             // TMA loads before they arrived on a_full, so a tile inside the stage is complete once a_full is;
             // a tile in a slot has a barrier of its own.
-            //
-            // With 32-token tiles a K block is 4 or 8 short MMAs, and a wait, an MMA batch and the commits each
-            // cost this warp 150-200 cycles of latency (850-900 cycles per K block were measured when they ran
-            // one after the other, more than the planes take to arrive).  So the barriers of block i + 1 are
-            // PROBED (test_wait, which never suspends) before the MMAs of block i are issued, and only a block
-            // that was not ready by then is waited for.
             int s = 0, xslot = 0;
             uint32_t xparity = 0, cnt0 = 0, cnt1 = 0;   // K blocks taken from each zip group so far
-            auto a_slot_of = [&](int stage, uint32_t& a_parity) -> int {
+            for (int i = 0; i < num_kb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1) {
                 constexpr int g0_slots = (kTotalSlots + 1) / 2, g1_slots = kTotalSlots / 2;   // 1 or 2 each
-                if ((stage & 1) == 0) {
+                int a;
+                uint32_t a_parity;
+                if ((s & 1) == 0) {
+                    a = g0_slots == 2 ? 2 * (int)(cnt0 & 1u) : 0;
                     a_parity = (g0_slots == 2 ? cnt0 >> 1 : cnt0) & 1u;
-                    return g0_slots == 2 ? 2 * (int)(cnt0 & 1u) : 0;
+                    ++cnt0;
+                } else {
+                    a = g1_slots == 2 ? 1 + 2 * (int)(cnt1 & 1u) : 1;
+                    a_parity = (g1_slots == 2 ? cnt1 >> 1 : cnt1) & 1u;
+                    ++cnt1;
                 }
-                a_parity = (g1_slots == 2 ? cnt1 >> 1 : cnt1) & 1u;
-                return g1_slots == 2 ? 1 + 2 * (int)(cnt1 & 1u) : 1;
-            };
-            uint32_t a_parity = 0;
-            int a = a_slot_of(0, a_parity);
-            DPS_STAMP(1, 0);
-            if (num_kb > 0) {
-                ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
-                DPS_CTA_STAMP_T(11, 32);
-                if (kXS && ok) ok = mbar_wait(smem_u32(&bar_x_full[0]), 0u);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                DPS_CTA_STAMP_T(10, 32);
-            }
-            for (int i = 0; i < num_kb && ok; ++i) {
-                DPS_STAMP(2, i);
                 const uint32_t xbase = kXS ? smem_base + (uint32_t)prm.x_offset + (uint32_t)(xslot * kXBytes)
                                            : smem_base + (uint32_t)s * kStage + kXOffset;
-                // block i is taken: advance the group's count, then look at block i + 1
-                if ((s & 1) == 0) ++cnt0; else ++cnt1;
-                const int s1 = (s + 1 == num_stages) ? 0 : s + 1;
-                int xslot1 = xslot;
-                uint32_t xparity1 = xparity;
-                if (kXS) {
-                    xslot1 = (xslot + 1 == kXS) ? 0 : xslot + 1;
-                    xparity1 ^= (xslot1 == 0);
-                }
-                uint32_t a1_parity = 0;
-                const int a1 = a_slot_of(s1, a1_parity);
-                bool next_ready = false;
-                if (i + 1 < num_kb) {
-                    next_ready = mbar_test_wait(smem_u32(&bar_a_full[a1]), a1_parity);
-                    if (kXS) next_ready = mbar_test_wait(smem_u32(&bar_x_full[xslot1]), xparity1) && next_ready;
-                }
+                DPS_STAMP(1, i);
+                ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
+                if (i == 0) DPS_CTA_STAMP_T(11, 32);
+                DPS_STAMP(9, i);
+                if (kXS && ok) ok = mbar_wait(smem_u32(&bar_x_full[xslot]), xparity);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                DPS_STAMP(2, i);
+                if (i == 0) DPS_CTA_STAMP_T(10, 32);
                 tc_fence_after_sync();
                 if (elect_one()) {
 #pragma unroll
@@ -665,17 +644,10 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 }
                 __syncwarp();
                 DPS_STAMP(3, i);
-                if (i + 1 < num_kb) {
-                    next_ready = __all_sync(0xFFFFFFFFu, next_ready);
-                    if (!next_ready) {
-                        DPS_STAMP(1, i + 1);
-                        ok = mbar_wait(smem_u32(&bar_a_full[a1]), a1_parity);
-                        DPS_STAMP(9, i + 1);
-                        if (kXS && ok) ok = mbar_wait(smem_u32(&bar_x_full[xslot1]), xparity1);
-                        ok = __all_sync(0xFFFFFFFFu, ok);
-                    }
+                if (kXS) {
+                    xslot = (xslot + 1 == kXS) ? 0 : xslot + 1;
+                    xparity ^= (xslot == 0);
                 }
-                s = s1; a = a1; xslot = xslot1; xparity = xparity1;
             }
         }
     } else {
