@@ -58,9 +58,20 @@ constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
 #ifndef DPS_RB2_FAST_BK
 #define DPS_RB2_FAST_BK 128
 #endif
+// Full-mode tiles of up to 64 tokens read 64 columns per K block (two planes: the stage is as large as a
+// fast-mode one), except the 32-token decode tiles: their stages are handed back as soon as the zip warps have
+// read them, so two stages of 128-byte rows do, and 128-byte rows stream better than 64-byte ones (measured at
+// 32 tokens, full mode, Llama-7B QKV / gate-up / o / down: 22.3 / 36.3 / 11.0 / 19.7 us against 22.8 / 38.9 /
+// 11.5 / 20.2).
+#ifndef DPS_FULL_BK128_MAX_TN
+#define DPS_FULL_BK128_MAX_TN 32
+#endif
+#ifndef DPS_FULL_BK128_MIN_TN
+#define DPS_FULL_BK128_MIN_TN 32
+#endif
 __host__ __device__ constexpr int block_k(bool full, int tn, int rb = 1) {
     if (rb == 2) return (full || tn > 128) ? 64 : DPS_RB2_FAST_BK;   // two accumulators of tn columns + four A slots in 512
-    return (tn >= DPS_BK64_FROM || (full && tn <= 64)) ? 64 : 128;
+    return (tn >= DPS_BK64_FROM || (full && tn <= 64 && !(tn >= DPS_FULL_BK128_MIN_TN && tn <= DPS_FULL_BK128_MAX_TN))) ? 64 : 128;
 }
 // Widest tile whose split-K partial sums are pushed into a mailbox of their own; wider tiles keep
 // the shared memory for the ring and pull the partial tiles out of it afterwards.
@@ -103,7 +114,7 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
 // registers and hand the stage back at once, the MMAs read the activations several K blocks later -- and a
 // tile fetched by the copy engine was measured to arrive 2000-2400 cycles after its request even out of L2.
 // So the tiles get slots of their own, requested as soon as the MMAs that read a slot last are complete,
-// five K blocks ahead (three were 2-4 % slower on most Llama-7B shapes in both modes, six and eight leave
+// five K blocks ahead in fast mode (three were 2-4 % slower on most Llama-7B shapes, six and eight leave
 // too few plane stages in fast mode).  0 = the activation tile travels inside the stage.
 // Not for 64-token tiles: their activation tile is as large as a plane stage, and the slots would leave a
 // ring of two.  Not for 16-token tiles either: measured 2-6 % slower there.
@@ -114,16 +125,20 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
 #define DPS_XSLOT_MAX_TN 32
 #endif
 #ifndef DPS_XSLOTS
-#define DPS_XSLOTS 5
+#define DPS_XSLOTS 5        // fast mode
 #endif
-constexpr int kMaxXSlots = DPS_XSLOTS;
-__host__ __device__ constexpr int x_slots(bool grouped, int tn, int rb) {
-    return (!grouped && rb == 1 && tn >= DPS_XSLOT_MIN_TN && tn <= DPS_XSLOT_MAX_TN) ? kMaxXSlots : 0;
+#ifndef DPS_XSLOTS_FULL
+#define DPS_XSLOTS_FULL 3   // full mode: a stage is two planes of 16 KB, and three 8 KB slots leave room for two
+#endif
+constexpr int kMaxXSlots = DPS_XSLOTS > DPS_XSLOTS_FULL ? DPS_XSLOTS : DPS_XSLOTS_FULL;
+__host__ __device__ constexpr int x_slots(bool full, bool grouped, int tn, int rb) {
+    return (!grouped && rb == 1 && tn >= DPS_XSLOT_MIN_TN && tn <= DPS_XSLOT_MAX_TN) ? (full ? DPS_XSLOTS_FULL : DPS_XSLOTS)
+                                                                                    : 0;
 }
 __host__ __device__ constexpr int x_tile_bytes(bool full, int tn, int rb = 1) { return tn * block_k(full, tn, rb) * 2; }
 // Bytes of one ring stage: planes and activations, or planes alone when the activations have slots.
 __host__ __device__ constexpr int ring_stage_bytes(bool full, int tn, bool grouped, int rb = 1) {
-    return stage_bytes(full, tn, rb) - (x_slots(grouped, tn, rb) ? x_tile_bytes(full, tn, rb) : 0);
+    return stage_bytes(full, tn, rb) - (x_slots(full, grouped, tn, rb) ? x_tile_bytes(full, tn, rb) : 0);
 }
 
 // Optional timeline trace (compile with -DDPS_TRACE): lane 0 of each role of CTA (0,0,0) stamps
@@ -312,7 +327,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
     constexpr int kStage = ring_stage_bytes(FULL, TN, GROUPED, RB);
     constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
-    constexpr int kXS = x_slots(GROUPED, TN, RB);          // 0 or 3
+    constexpr int kXS = x_slots(FULL, GROUPED, TN, RB);    // 0, or the slots of this mode
     constexpr int kXBytes = x_tile_bytes(FULL, TN, RB);
     constexpr uint32_t kCols = tmem_cols(FULL, TN, RB);
     static_assert(RB == 1 || RB == 2, "one or two row blocks per CTA");
@@ -924,7 +939,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     constexpr int kZipGroups = zip_groups(FULL, TN);
     constexpr int kZipThreads = kZipGroups * 128;
     constexpr int kTotalSlots = a_slots_max(FULL, TN);
-    static_assert(x_slots(GROUPED, TN, RB) == 0, "the persistent kernel keeps activations in the stages");
+    static_assert(x_slots(FULL, GROUPED, TN, RB) == 0, "the persistent kernel keeps activations in the stages");
     static_assert(TN % kEpiChunkCols == 0, "tiles are drained 32 token columns at a time");
 
     extern __shared__ uint8_t smem_raw[];
@@ -1392,7 +1407,7 @@ template <int ENC, bool FULL, int TN>
 cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y, int64_t M, int64_t N, int64_t K,
                       int* status, cudaStream_t stream) {
     constexpr int kStage = ring_stage_bytes(FULL, TN, false);   // planes only when the activations have slots
-    constexpr int kXRing = x_slots(false, TN, 1) * x_tile_bytes(FULL, TN);
+    constexpr int kXRing = x_slots(FULL, false, TN, 1) * x_tile_bytes(FULL, TN);
     constexpr int kZipGroups = zip_groups(FULL, TN);
     constexpr int kThreads = cta_threads(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
