@@ -116,8 +116,7 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
 // So the tiles get slots of their own, requested as soon as the MMAs that read a slot last are complete,
 // five K blocks ahead in fast mode (three were 2-4 % slower on most Llama-7B shapes, six and eight leave
 // too few plane stages in fast mode).  0 = the activation tile travels inside the stage.
-// Not for 64-token tiles: their activation tile is as large as a plane stage, and the slots would leave a
-// ring of two.  Not for 16-token tiles either: measured 2-6 % slower there.
+// Not for 16-token tiles: measured 2-6 % slower there.
 #ifndef DPS_XSLOT_MIN_TN
 #define DPS_XSLOT_MIN_TN 32
 #endif
@@ -130,10 +129,20 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
 #ifndef DPS_XSLOTS_FULL
 #define DPS_XSLOTS_FULL 3   // full mode: a stage is two planes of 16 KB, and three 8 KB slots leave room for two
 #endif
-constexpr int kMaxXSlots = DPS_XSLOTS > DPS_XSLOTS_FULL ? DPS_XSLOTS : DPS_XSLOTS_FULL;
+constexpr int kMaxXSlots = 8;   // barrier array size
+// 64-token tiles: the split-K mailbox takes 36 KB there, which leaves three plane stages and three slots in
+// full mode and two of each in fast mode (one more slot each no longer fits two CTAs on an SM).  Measured
+// at 64 tokens on the Llama-7B shapes against tiles that carry the activations in the stages: 0-14 % faster.
+#ifndef DPS_XSLOTS_FULL64
+#define DPS_XSLOTS_FULL64 3
+#endif
+#ifndef DPS_XSLOTS_FAST64
+#define DPS_XSLOTS_FAST64 2
+#endif
 __host__ __device__ constexpr int x_slots(bool full, bool grouped, int tn, int rb) {
-    return (!grouped && rb == 1 && tn >= DPS_XSLOT_MIN_TN && tn <= DPS_XSLOT_MAX_TN) ? (full ? DPS_XSLOTS_FULL : DPS_XSLOTS)
-                                                                                    : 0;
+    if (grouped || rb != 1) return 0;
+    if (tn == 64) return full ? DPS_XSLOTS_FULL64 : DPS_XSLOTS_FAST64;
+    return (tn >= DPS_XSLOT_MIN_TN && tn <= DPS_XSLOT_MAX_TN) ? (full ? DPS_XSLOTS_FULL : DPS_XSLOTS) : 0;
 }
 __host__ __device__ constexpr int x_tile_bytes(bool full, int tn, int rb = 1) { return tn * block_k(full, tn, rb) * 2; }
 // Bytes of one ring stage: planes and activations, or planes alone when the activations have slots.
