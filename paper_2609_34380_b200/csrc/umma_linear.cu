@@ -144,6 +144,14 @@ __host__ __device__ constexpr int x_slots(bool full, bool grouped, int tn, int r
     if (tn == 64) return full ? DPS_XSLOTS_FULL64 : DPS_XSLOTS_FAST64;
     return (tn >= DPS_XSLOT_MIN_TN && tn <= DPS_XSLOT_MAX_TN) ? (full ? DPS_XSLOTS_FULL : DPS_XSLOTS) : 0;
 }
+// Slots of a launch whose K is not split (no mailbox in shared memory): what the freed space holds best.
+// 64-token tiles, fast mode: three slots and three stages instead of two and four (gate-up at 64 tokens:
+// 22.3 us against 25.1); full mode: five slots beside the same number of stages.
+__host__ __device__ constexpr int x_slots_alone(bool full, int tn) {
+    if (x_slots(full, false, tn, 1) == 0) return 0;
+    if (tn == 64) return full ? 5 : 3;
+    return 5;
+}
 __host__ __device__ constexpr int x_tile_bytes(bool full, int tn, int rb = 1) { return tn * block_k(full, tn, rb) * 2; }
 // Bytes of one ring stage: planes and activations, or planes alone when the activations have slots.
 __host__ __device__ constexpr int ring_stage_bytes(bool full, int tn, bool grouped, int rb = 1) {
@@ -200,6 +208,7 @@ struct UmmaParams {
     int split;       // K split = cluster size along z; partial tiles are summed through DSMEM
     int red_offset;  // byte offset (from the aligned base of dynamic smem) of the split-K mailbox
     int x_offset;    // byte offset of the activation slots (tiles whose activations do not ride in the stages)
+    int x_slots;     // activation slots (tiles that keep the activations apart from the plane ring)
     int pair_min;    // ring depth from which stages are filled two at a time
     int tail_parts;  // persistent dense launches: the tiles of the last, partial round are cut into this many
                      // token ranges (1, 2 or 4), each a work item of its own
@@ -336,7 +345,8 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
     constexpr int kPlaneStageBytes = plane_stage_bytes(FULL, TN, RB);
     constexpr int kStage = ring_stage_bytes(FULL, TN, GROUPED, RB);
     constexpr int kXOffset = kPlaneStageBytes * (FULL ? 2 : 1);
-    constexpr int kXS = x_slots(FULL, GROUPED, TN, RB);    // 0, or the slots of this mode
+    constexpr bool kXS = x_slots(FULL, GROUPED, TN, RB) > 0;   // the activations have slots of their own ...
+    const int xs_n = prm.x_slots;                               // ... this many (chosen per launch: what fits)
     constexpr int kXBytes = x_tile_bytes(FULL, TN, RB);
     constexpr uint32_t kCols = tmem_cols(FULL, TN, RB);
     static_assert(RB == 1 || RB == 2, "one or two row blocks per CTA");
@@ -479,7 +489,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             for (int t = 0; t < kXAtoms; ++t)
                 tma_load_2d(dst + kXOffset + (uint32_t)(t * TN * 128), &map_x, full, k + t * 64, m0);
         };
-        auto load_x_slot = [&](int j, int slot) {   // activation tile of K block j into its own slot (j % kXS)
+        auto load_x_slot = [&](int j, int slot) {   // activation tile of K block j into its own slot
             const uint32_t full = smem_u32(&bar_x_full[slot]);
             const uint32_t dst = smem_base + (uint32_t)prm.x_offset + (uint32_t)(slot * kXBytes);
             const int k = (rank + j * split) * kBlockK;
@@ -561,12 +571,12 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                     dep = true;
                 }
                 if (dep && ix < num_kb &&
-                    (ix < kXS || __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_x_empty[sx]), phx)))) {
+                    (ix < xs_n || __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_x_empty[sx]), phx)))) {
                     if (elect_one()) load_x_slot(ix, sx);
                     __syncwarp();
                     ++ix;
-                    sx = (sx + 1 == kXS) ? 0 : sx + 1;
-                    if (sx == 0 && ix > kXS) phx ^= 1u;
+                    sx = (sx + 1 == xs_n) ? 0 : sx + 1;
+                    if (sx == 0 && ix > xs_n) phx ^= 1u;
                     progress = true;
                 }
                 if (progress) {
@@ -621,7 +631,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             }
         } else {
             // Stage s belongs to zip group s % 2, which rotates through its own A slots (see zip_blocks); the
-            // activation tile rides in the stage or sits in slot i % kXS.  The zip warps waited for the stage's
+            // activation tile rides in the stage or sits in a slot of its own (K block i: slot i % slots).  The zip warps waited for the stage's
             // TMA loads before they arrived on a_full, so a tile inside the stage is complete once a_full is;
             // a tile in a slot has a barrier of its own.
             int s = 0, xslot = 0;
@@ -669,7 +679,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 __syncwarp();
                 DPS_STAMP(3, i);
                 if (kXS) {
-                    xslot = (xslot + 1 == kXS) ? 0 : xslot + 1;
+                    xslot = (xslot + 1 == xs_n) ? 0 : xslot + 1;
                     xparity ^= (xslot == 0);
                 }
             }
@@ -700,7 +710,7 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
                 ok = e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst);
         } else {
             ZipState zst;
-            ok = zip_blocks<ENC, FULL, TN, RB, (kXS > 0)>(zc, zst);
+            ok = zip_blocks<ENC, FULL, TN, RB, kXS>(zc, zst);
         }
         // E4M3 fast mode multiplied with 2^8 times the weights (hardware FP8 conversion)
         const float out_scale = (!FULL && !e5m2) ? 0.00390625f : 1.0f;
@@ -1416,7 +1426,9 @@ template <int ENC, bool FULL, int TN>
 cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y, int64_t M, int64_t N, int64_t K,
                       int* status, cudaStream_t stream) {
     constexpr int kStage = ring_stage_bytes(FULL, TN, false);   // planes only when the activations have slots
-    constexpr int kXRing = x_slots(FULL, false, TN, 1) * x_tile_bytes(FULL, TN);
+    constexpr int kXSlots = x_slots(FULL, false, TN, 1);            // with a split-K mailbox in shared memory
+    constexpr int kXSlotsAlone = x_slots_alone(FULL, TN);           // without one (K not split)
+    constexpr int kXTile = x_tile_bytes(FULL, TN);
     constexpr int kZipGroups = zip_groups(FULL, TN);
     constexpr int kThreads = cta_threads(FULL, TN);
     constexpr int kCtasPerSm = tmem_cols(FULL, TN) <= 256 ? 2 : 1;
@@ -1437,12 +1449,13 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
         return e ? atoi(e) : 8;
     }();
     auto ring_depth = [&](int mail_bytes) {
-        int d = (smem_total - mail_bytes - kXRing) / kStage;
+        const int x_ring = (mail_bytes > 0 ? kXSlots : kXSlotsAlone) * kXTile;
+        int d = (smem_total - mail_bytes - x_ring) / kStage;
         if (d > max_stages) d = max_stages;
         if (d < 2) d = 2;
         return d;
     };
-    const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kXRing + kMailMax + 1024;
+    const size_t smem_query = (size_t)ring_depth(kMailMax) * kStage + kXSlots * kXTile + kMailMax + 1024;
     auto kernel = umma_linear_kernel<ENC, FULL, TN, false>;
     // CTAs that can be resident at once for each cluster size: per instantiation and per device, filled by
     // the first call on that device and read only after that set-up has returned.
@@ -1524,7 +1537,9 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     const int slots = split > 1 ? (TN + split - 1) / split : 0;
     const int mail_bytes = (split > 1 && kMailMax > 0) ? split * slots * kTileRows * 4 : 0;
     const int stages = ring_depth(mail_bytes);
-    const size_t smem = (size_t)stages * kStage + kXRing + mail_bytes + 1024;
+    const int xs_n = mail_bytes > 0 ? kXSlots : kXSlotsAlone;
+    const int x_ring = xs_n * kXTile;
+    const size_t smem = (size_t)stages * kStage + x_ring + mail_bytes + 1024;
     if (kMailMax == 0 && (size_t)stages * kStage < (size_t)TN * kTileRows * 4) split = 1;  // pull mode overlays the ring
     if (getenv("DPS_DEBUG"))
         fprintf(stderr, "[dps] umma TN=%d full=%d N=%lld K=%lld M=%lld stages=%d split=%d capacity=%d,%d,%d,%d,%d,%d,%d,%d\n",
@@ -1545,7 +1560,8 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     prm.num_stages = stages;
     prm.split = split;
     prm.x_offset = stages * kStage;
-    prm.red_offset = stages * kStage + kXRing;
+    prm.x_slots = xs_n;
+    prm.red_offset = stages * kStage + x_ring;
     prm.status = status;
     prm.pair_min = pair_min_depth();
 #ifdef DPS_TRACE
