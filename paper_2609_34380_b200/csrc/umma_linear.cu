@@ -67,7 +67,7 @@ constexpr int kTileRows = 128;   // weight rows per CTA (UMMA M)
 #define DPS_FULL_BK128_MAX_TN 32
 #endif
 #ifndef DPS_FULL_BK128_MIN_TN
-#define DPS_FULL_BK128_MIN_TN 32
+#define DPS_FULL_BK128_MIN_TN 16   // 16-token tiles alike: 21.3 / 36.1 / 18.8 us against 23.0 / 38.4 / 20.0 (no o: too small)
 #endif
 __host__ __device__ constexpr int block_k(bool full, int tn, int rb = 1) {
     if (rb == 2) return (full || tn > 128) ? 64 : DPS_RB2_FAST_BK;   // two accumulators of tn columns + four A slots in 512
@@ -116,7 +116,7 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
 // So the tiles get slots of their own, requested as soon as the MMAs that read a slot last are complete,
 // five K blocks ahead in fast mode (three were 2-4 % slower on most Llama-7B shapes, six and eight leave
 // too few plane stages in fast mode).  0 = the activation tile travels inside the stage.
-// Not for 16-token tiles: measured 2-6 % slower there.
+// (16- and 64-token tiles: below.)
 #ifndef DPS_XSLOT_MIN_TN
 #define DPS_XSLOT_MIN_TN 32
 #endif
@@ -133,6 +133,10 @@ constexpr int kMaxXSlots = 8;   // barrier array size
 // 64-token tiles: the split-K mailbox takes 36 KB there, which leaves three plane stages and three slots in
 // full mode and two of each in fast mode (one more slot each no longer fits two CTAs on an SM).  Measured
 // at 64 tokens on the Llama-7B shapes against tiles that carry the activations in the stages: 0-14 % faster.
+// 16-token tiles: slots in full mode only (fast mode with slots: gate-up 1-3 % faster, down 4 % slower).
+#ifndef DPS_XSLOTS_FAST16
+#define DPS_XSLOTS_FAST16 0
+#endif
 #ifndef DPS_XSLOTS_FULL64
 #define DPS_XSLOTS_FULL64 3
 #endif
@@ -142,6 +146,7 @@ constexpr int kMaxXSlots = 8;   // barrier array size
 __host__ __device__ constexpr int x_slots(bool full, bool grouped, int tn, int rb) {
     if (grouped || rb != 1) return 0;
     if (tn == 64) return full ? DPS_XSLOTS_FULL64 : DPS_XSLOTS_FAST64;
+    if (tn == 16) return full ? DPS_XSLOTS_FULL : DPS_XSLOTS_FAST16;
     return (tn >= DPS_XSLOT_MIN_TN && tn <= DPS_XSLOT_MAX_TN) ? (full ? DPS_XSLOTS_FULL : DPS_XSLOTS) : 0;
 }
 // Slots of a launch whose K is not split (no mailbox in shared memory): what the freed space holds best.
