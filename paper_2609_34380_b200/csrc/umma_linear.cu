@@ -157,6 +157,28 @@ __host__ __device__ constexpr int x_slots_alone(bool full, int tn) {
     if (tn == 64) return full ? 5 : 3;
     return 5;
 }
+// The persistent kernel keeps the activations of GROUPED launches in slots as well: an MoE layer streams its
+// planes once, three or four 56 KB stages of planes + activations per SM left the stream waiting for the ring
+// (two stages instead of three: 25 % slower), and a plane stage is free again as soon as the zip warps have
+// read it, while its activation tile has to stay until the MMAs are complete.  Dense persistent launches
+// (prefill) are bound by the tensor pipe, not by the ring: their activations stay in the stages.
+#ifndef DPS_PERSIST_XSLOTS
+#define DPS_PERSIST_XSLOTS 4   // measured on Mixtral expert layers, 96-token tiles: 3 slots 3-5 % slower, 5 up to 13 %
+#endif
+__host__ __device__ constexpr int persist_x_slots(bool grouped) { return grouped ? DPS_PERSIST_XSLOTS : 0; }
+// ... and with two row blocks they have two MMA-issuing warps, one per row block (the CTA's last warp is the
+// second).  Per-K-block stamps of a fast-mode Mixtral gate/up layer (96-token tiles, 16 MMAs of 48 cycles per
+// K block): one warp spent 1240 cycles per block, 470 of them on its waits and commits with the tensor pipe
+// running dry behind them; with two issuers one warp's waits hide behind the other's MMAs.
+#ifndef DPS_PERSIST_TWO_MMA
+#define DPS_PERSIST_TWO_MMA 1
+#endif
+__host__ __device__ constexpr bool persist_two_mma(bool grouped, int rb) {
+    return DPS_PERSIST_TWO_MMA != 0 && persist_x_slots(grouped) > 0 && rb == 2;
+}
+__host__ __device__ constexpr int persist_threads(bool full, int tn, bool grouped, int rb) {
+    return cta_threads(full, tn) + (persist_two_mma(grouped, rb) ? 32 : 0);
+}
 __host__ __device__ constexpr int x_tile_bytes(bool full, int tn, int rb = 1) { return tn * block_k(full, tn, rb) * 2; }
 // Bytes of one ring stage: planes and activations, or planes alone when the activations have slots.
 __host__ __device__ constexpr int ring_stage_bytes(bool full, int tn, bool grouped, int rb = 1) {
@@ -947,7 +969,7 @@ __device__ __forceinline__ TileCoords tile_coords(int lin, int part, int parts, 
 }
 
 template <int ENC, bool FULL, int TN, bool GROUPED, int RB>
-__global__ void __launch_bounds__(cta_threads(FULL, TN), 1)
+__global__ void __launch_bounds__(persist_threads(FULL, TN, GROUPED, RB), 1)
 umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_constant__ CUtensorMap map_r,
                        const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_x2,
                        const __grid_constant__ CUtensorMap map_x4, const UmmaParams prm, const GroupedParams gp) {
@@ -963,7 +985,12 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     constexpr int kZipGroups = zip_groups(FULL, TN);
     constexpr int kZipThreads = kZipGroups * 128;
     constexpr int kTotalSlots = a_slots_max(FULL, TN);
-    static_assert(x_slots(FULL, GROUPED, TN, RB) == 0, "the persistent kernel keeps activations in the stages");
+    constexpr bool kXS = persist_x_slots(GROUPED) > 0;        // the activations have slots of their own ...
+    constexpr int kRing = kXS ? kXOffset : kStage;            // ... and a ring stage holds planes only
+    constexpr bool kTwoMma = persist_two_mma(GROUPED, RB);    // one MMA warp per row block
+    constexpr int kMmaWarps = kTwoMma ? 2 : 1;
+    constexpr int kZipEnd = 2 + 4 * zip_groups(FULL, TN);     // first warp behind the zip warps
+    constexpr int kXBytes = x_tile_bytes(FULL, TN, RB);
     static_assert(TN % kEpiChunkCols == 0, "tiles are drained 32 token columns at a time");
 
     extern __shared__ uint8_t smem_raw[];
@@ -973,6 +1000,8 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     __shared__ __align__(8) uint64_t bar_a_empty[kMaxAStages];
     __shared__ __align__(8) uint64_t bar_d_full;
     __shared__ __align__(8) uint64_t bar_d_empty;
+    __shared__ __align__(8) uint64_t bar_x_full[kMaxXSlots];
+    __shared__ __align__(8) uint64_t bar_x_empty[kMaxXSlots];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ int s_rows[GROUPED ? TN : 1];   // grouped launches: row ids of the current tile's tokens
@@ -989,13 +1018,18 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     if (threadIdx.x == 0) {
         for (int s = 0; s < num_stages; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
-            mbar_init(smem_u32(&bar_empty[s]), RB == 2 ? 9 : 5);
+            // the zip warps that read the stage, and the tcgen05.commit if the activations ride in it
+            mbar_init(smem_u32(&bar_empty[s]), (RB == 2 ? 8 : 4) + (kXS ? 0 : 1));
         }
         for (int a = 0; a < kMaxAStages; ++a) {
             mbar_init(smem_u32(&bar_a_full[a]), 4);
             mbar_init(smem_u32(&bar_a_empty[a]), 1);
         }
-        mbar_init(smem_u32(&bar_d_full), 1);
+        for (int a = 0; a < kMaxXSlots; ++a) {
+            mbar_init(smem_u32(&bar_x_full[a]), 1);
+            mbar_init(smem_u32(&bar_x_empty[a]), kMmaWarps);   // one tcgen05.commit per MMA warp
+        }
+        mbar_init(smem_u32(&bar_d_full), kMmaWarps);
         mbar_init(smem_u32(&bar_d_empty), kZipGroups * 4);   // one arrival per zip warp
         abort_flag = 0;
         fence_barrier_init();
@@ -1029,9 +1063,87 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
     int last_ncols = 0, last_n0 = 0, last_m0 = 0;   // the K-half item's tile, for the pair's reduction below
     if (warp == 0) {
         // ---------------- TMA producer ----------------
+        if (kXS) {
+            // Two streams over the same sequence of (work item, K block): planes into the ring, activation
+            // tiles into their slots.  A stage is free when the zip warps have read it, a slot when the MMAs
+            // that read it are complete; the loop probes (test_wait never suspends) whichever barrier is next
+            // in each stream, so neither waits for the other's consumer.  The clock keeps the wait bounded.
+            struct Cursor {
+                int step = 0, i = 0, nkb = 0, kb0 = 0, row0 = 0, m0 = 0;
+                bool live = false, done = false;
+            };
+            auto advance = [&](Cursor& c) {      // to the next K block of the stream, fetching work items as needed
+                if (c.live && ++c.i < c.nkb) return;
+                c.live = false;
+                while (!c.done && !c.live) {
+                    int l, pt, kh;
+                    if (!next_work(c.step, t_main, total, parts, ksplit, l, pt, kh)) { c.done = true; break; }
+                    ++c.step;
+                    const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(l, pt, parts, row_tiles, tok_tiles, prm, gp);
+                    if (t.tile_tokens <= 0) continue;
+                    c.kb0 = kh == 1 ? num_kb / 2 : 0;
+                    c.nkb = kh < 0 ? num_kb : (kh == 0 ? num_kb / 2 : num_kb - num_kb / 2);
+                    c.row0 = t.plane_row0;
+                    c.m0 = t.m0;
+                    c.i = 0;
+                    c.live = c.nkb > 0;
+                }
+            };
+            Cursor cp, cx;
+            advance(cp);
+            advance(cx);
+            int sp = 0, sx = 0;
+            uint32_t php = 0, phx = 0;
+            uint32_t idle = 0;
+            unsigned long long t0 = 0;
+            const int xs_n = prm.x_slots;
+            while ((cp.live || cx.live) && ok) {
+                bool progress = false;
+                // (a fresh barrier passes a wait for the phase before its first at once)
+                if (cp.live && __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_empty[sp]), php ^ 1u))) {
+                    if (elect_one()) {
+                        const uint32_t full = smem_u32(&bar_full[sp]);
+                        const uint32_t dst = smem_base + (uint32_t)sp * kRing;
+                        const int k = (cp.kb0 + cp.i) * kBlockK;
+                        DPS_STAMP(0, cp.i);
+                        mbar_arrive_expect_tx(full, (uint32_t)kRing);
+                        tma_load_2d(dst, &map_p, full, k, cp.row0);
+                        if (FULL) tma_load_2d(dst + kPlaneStageBytes, &map_r, full, k, cp.row0);
+                    }
+                    __syncwarp();
+                    advance(cp);
+                    sp = (sp + 1 == num_stages) ? 0 : sp + 1;
+                    php ^= (sp == 0);
+                    progress = true;
+                }
+                if (cx.live && __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_x_empty[sx]), phx ^ 1u))) {
+                    if (elect_one()) {
+                        const uint32_t full = smem_u32(&bar_x_full[sx]);
+                        const uint32_t dst = smem_base + (uint32_t)prm.x_offset + (uint32_t)(sx * kXBytes);
+                        const int k = (cx.kb0 + cx.i) * kBlockK;
+                        mbar_arrive_expect_tx(full, (uint32_t)kXBytes);
+#pragma unroll
+                        for (int a = 0; a < kXAtoms; ++a)
+                            tma_load_2d(dst + (uint32_t)(a * TN * 128), &map_x, full, k + a * 64, cx.m0);
+                    }
+                    __syncwarp();
+                    advance(cx);
+                    sx = (sx + 1 == xs_n) ? 0 : sx + 1;
+                    phx ^= (sx == 0);
+                    progress = true;
+                }
+                if (progress) {
+                    idle = 0;
+                } else if ((++idle & 1023u) == 0) {
+                    const unsigned long long now = global_timer_ns();
+                    if (idle == 1024u) t0 = now;
+                    else if (now - t0 > kWaitLimitNs) ok = false;
+                }
+            }
+        }
         int s = 0;
         uint32_t ph = 0;
-        for (int step = 0; ok && next_work(step, t_main, total, parts, ksplit, lin, part, khalf); ++step) {
+        for (int step = 0; !kXS && ok && next_work(step, t_main, total, parts, ksplit, lin, part, khalf); ++step) {
             const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
             if (t.tile_tokens <= 0) continue;
             const CUtensorMap* xmap = t.parts == 4 ? &map_x4 : t.parts == 2 ? &map_x2 : &map_x;
@@ -1056,11 +1168,15 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                 __syncwarp();
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
+    } else if (warp == 1 || (kTwoMma && warp == kZipEnd)) {
+        // ---------------- MMA issuer (one, or one per row block) ----------------
+        const int w = warp == 1 ? 0 : 1;
         int s = 0;
         int cnt[2] = {0, 0};
         int it = 0;
+        int xslot = 0;            // activation slot of the next K block (launches with activation slots)
+        uint32_t xparity = 0;
+        const int xs_n = prm.x_slots;
         for (int step = 0; ok && next_work(step, t_main, total, parts, ksplit, lin, part, khalf); ++step) {
             const TileCoords t = tile_coords<ENC, TN, GROUPED, RB>(lin, part, parts, row_tiles, tok_tiles, prm, gp);
             if (t.tile_tokens <= 0) continue;
@@ -1075,9 +1191,18 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                 tc_fence_after_sync();
             }
             for (int i = 0; i < nkb && ok; ++i, s = (s + 1 == num_stages) ? 0 : s + 1) {
-                const uint32_t xbase = smem_base + (uint32_t)s * kStage + kXOffset;
+                const uint32_t xbase = kXS ? smem_base + (uint32_t)prm.x_offset + (uint32_t)(xslot * kXBytes)
+                                           : smem_base + (uint32_t)s * kStage + kXOffset;
+                DPS_STAMP(1, i);
+                if (kXS) {
+                    ok = mbar_wait(smem_u32(&bar_x_full[xslot]), xparity);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                }
+                DPS_STAMP(9, i);
 #pragma unroll
                 for (int rb = 0; rb < RB; ++rb) {
+                    if (kTwoMma && rb != w) continue;
                     // RB == 2: zip group rb serves row block rb of every K block; RB == 1: group s % 2
                     const int g = RB == 2 ? rb : (s & 1);
                     const int g_slots = RB == 2 ? 2 : (kTotalSlots - g + 1) / 2;
@@ -1088,6 +1213,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                     ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
+                    if (rb == 0) DPS_STAMP(2, i); else DPS_STAMP(10, i);
                     tc_fence_after_sync();
                     if (elect_one()) {
 #pragma unroll
@@ -1098,17 +1224,23 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                                         idesc, (i > 0 || j > 0) ? 1u : 0u);
                         }
                         umma_commit(smem_u32(&bar_a_empty[a]));
-                        if (rb == RB - 1) {
-                            umma_commit(smem_u32(&bar_empty[s]));
+                        if (kTwoMma || rb == RB - 1) {
+                            if (kXS) umma_commit(smem_u32(&bar_x_empty[xslot]));   // the slot may be refilled ...
+                            else umma_commit(smem_u32(&bar_empty[s]));             // ... or the stage with the tile
                             if (i == nkb - 1) umma_commit(smem_u32(&bar_d_full));
                         }
                     }
                     __syncwarp();
                 }
+                DPS_STAMP(3, i);
+                if (kXS) {
+                    xslot = (xslot + 1 == xs_n) ? 0 : xslot + 1;
+                    xparity ^= (xslot == 0);
+                }
             }
             ++it;
         }
-    } else {
+    } else if (warp < kZipEnd) {
         // ---------------- zip warps: planes -> FP16 -> tensor memory; then the tile's epilogue ----------------
         const int group = (warp - 2) >> 2;
         const int q = warp & 3;
@@ -1117,7 +1249,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         const int zt = (int)threadIdx.x - 64;   // index among the zip threads
         ZipCtx zc;
         zc.group = group; zc.warp = warp; zc.lane = lane; zc.row = row;
-        zc.num_kb = num_kb; zc.num_stages = num_stages; zc.stage_bytes = kStage;
+        zc.num_kb = num_kb; zc.num_stages = num_stages; zc.stage_bytes = kRing;
         zc.smem_base = smem_base; zc.tmem_a = tmem_a; zc.lane_base = lane_base;
         zc.sw = kBlockK == 128 ? (uint32_t)(row & 7) : (uint32_t)((row >> 1) & 3);
         zc.bar_full = bar_full; zc.bar_empty = bar_empty; zc.bar_a_full = bar_a_full; zc.bar_a_empty = bar_a_empty;
@@ -1134,10 +1266,12 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
             if (ok) {
                 if (GROUPED && !(ENC == kEncE4M3 || ENC == kEncE5M2))
                     ok = (FULL && t.rounded)
-                             ? (t.e5m2 ? zip_blocks<kEncE5M2R, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3R, FULL, TN, RB>(zc, zst))
-                             : (t.e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB>(zc, zst) : zip_blocks<kEncE4M3, FULL, TN, RB>(zc, zst));
+                             ? (t.e5m2 ? zip_blocks<kEncE5M2R, FULL, TN, RB, kXS>(zc, zst)
+                                       : zip_blocks<kEncE4M3R, FULL, TN, RB, kXS>(zc, zst))
+                             : (t.e5m2 ? zip_blocks<kEncE5M2, FULL, TN, RB, kXS>(zc, zst)
+                                       : zip_blocks<kEncE4M3, FULL, TN, RB, kXS>(zc, zst));
                 else
-                    ok = zip_blocks<ENC, FULL, TN, RB>(zc, zst);
+                    ok = zip_blocks<ENC, FULL, TN, RB, kXS>(zc, zst);
             }
             const float out_scale = (!FULL && !t.e5m2) ? 0.00390625f : 1.0f;   // E4M3 fast mode carries 2^8
             if (ok) ok = mbar_wait(smem_u32(&bar_d_full), (uint32_t)it & 1u);
@@ -1235,7 +1369,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         // of a token (32 contiguous bytes each, two 16-byte loads from each partial tile)
         constexpr int kPieces = kRowsCta / 8;
         const int my_cols = (ncols - (int)rank + 1) / 2;
-        for (int idx = (int)threadIdx.x; idx < my_cols * kPieces; idx += cta_threads(FULL, TN)) {
+        for (int idx = (int)threadIdx.x; idx < my_cols * kPieces; idx += (int)blockDim.x) {
             const int c = (int)rank + 2 * (idx / kPieces), qq = idx % kPieces;
             const int n = n0 + qq * 8;
             if (n >= prm.N) continue;
@@ -1337,13 +1471,19 @@ template <int ENC, bool FULL, int TN, bool GROUPED, int RB>
 cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, const CUtensorMap& mx, UmmaParams prm,
                               const GroupedParams& gp, int64_t tiles, const void* x, int64_t x_rows,
                               cudaStream_t stream) {
-    constexpr int kStage = stage_bytes(FULL, TN, RB);
+    constexpr int kXSlots = persist_x_slots(GROUPED);
+    constexpr int kXTile = x_tile_bytes(FULL, TN, RB);
+    // a ring stage: planes and activations, or planes only when the activations have slots
+    constexpr int kStage = stage_bytes(FULL, TN, RB) - (kXSlots ? kXTile : 0);
     constexpr int kEpiBytes = kEpiChunkCols * kTileRows * RB * 2;
-    constexpr int kThreads = cta_threads(FULL, TN);
-    int stages = (216 * 1024 - kEpiBytes) / kStage;
+    constexpr int kThreads = persist_threads(FULL, TN, GROUPED, RB);
+    int xs_n = kXSlots;     // one slot fewer where that buys the third plane stage (128-token tiles, fast mode)
+    if (xs_n > 3 && (216 * 1024 - kEpiBytes - xs_n * kXTile) / kStage < 3) --xs_n;
+    int stages = (216 * 1024 - kEpiBytes - xs_n * kXTile) / kStage;
     if (stages > 8) stages = 8;
     if (stages < 2) stages = 2;
-    const size_t smem = (size_t)stages * kStage + kEpiBytes + 1024;
+    const size_t ring_bytes = (size_t)stages * kStage + (size_t)xs_n * kXTile;   // idle after a CTA's last item
+    const size_t smem = ring_bytes + kEpiBytes + 1024;
     auto kernel = umma_persistent_kernel<ENC, FULL, TN, GROUPED, RB>;
     static PerDeviceOnce setup;     // per instantiation and per device
     {
@@ -1356,8 +1496,9 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
         if (e != cudaSuccess) return e;
     }
     prm.num_stages = stages;
-    prm.red_offset = stages * kStage;   // the epilogue's chunk buffer
-    prm.x_offset = 0;
+    prm.red_offset = (int)ring_bytes;   // the epilogue's chunk buffer
+    prm.x_offset = stages * kStage;     // the activation slots, if any
+    prm.x_slots = xs_n;
     prm.pair_min = pair_min_depth();
     int64_t grid = tiles < sm_count() ? tiles : sm_count();
 
@@ -1371,10 +1512,9 @@ cudaError_t launch_persistent(const CUtensorMap& mp, const CUtensorMap& mr, cons
     const bool ksplit_enabled = ksplit_mode != 0;
     // Dense launches with at most half as many tiles as SMs: two CTAs per tile, each with one half of K
     // (the kernel treats all of them as the "last round").
-    if (!GROUPED && ksplit_mode == 1 && pair_all_tiles(tiles) &&
-        (size_t)TN * kTileRows * RB * 4 <= (size_t)stages * kStage)
+    if (!GROUPED && ksplit_mode == 1 && pair_all_tiles(tiles) && (size_t)TN * kTileRows * RB * 4 <= ring_bytes)
         grid = 2 * tiles;
-    const bool pairs = ksplit_enabled && grid >= 2 && (size_t)TN * kTileRows * RB * 4 <= (size_t)stages * kStage;
+    const bool pairs = ksplit_enabled && grid >= 2 && (size_t)TN * kTileRows * RB * 4 <= ring_bytes;
     if (pairs) grid &= ~(int64_t)1;
     prm.split = (pairs && ksplit_mode == 1) ? 2 : 1;
     // Last, partial round of a dense launch: cut its tiles into 2 or 4 token ranges if that gives
