@@ -166,15 +166,18 @@ __host__ __device__ constexpr int x_slots_alone(bool full, int tn) {
 #define DPS_PERSIST_XSLOTS 4   // measured on Mixtral expert layers, 96-token tiles: 3 slots 3-5 % slower, 5 up to 13 %
 #endif
 __host__ __device__ constexpr int persist_x_slots(bool grouped) { return grouped ? DPS_PERSIST_XSLOTS : 0; }
-// ... and with two row blocks they have two MMA-issuing warps, one per row block (the CTA's last warp is the
-// second).  Per-K-block stamps of a fast-mode Mixtral gate/up layer (96-token tiles, 16 MMAs of 48 cycles per
+// ... and tiles with two row blocks (grouped or dense) have two MMA-issuing warps, one per row block (the CTA's
+// last warp is the second; dense fast-mode prefill on 256 x 192 tiles: +4 %, 1.30 -> 1.35 and 1.34 -> 1.39 PFLOP/s
+// on Llama-7B QKV / gate-up at 2048 and 8192 tokens).  Probing the next K block's barriers before issuing the
+// MMAs of the current one, so that a wait on a barrier that completed long ago costs nothing, was measured
+// 3-5 % SLOWER on prefill in both modes and is not done.  Per-K-block stamps of a fast-mode Mixtral gate/up layer (96-token tiles, 16 MMAs of 48 cycles per
 // K block): one warp spent 1240 cycles per block, 470 of them on its waits and commits with the tensor pipe
 // running dry behind them; with two issuers one warp's waits hide behind the other's MMAs.
 #ifndef DPS_PERSIST_TWO_MMA
-#define DPS_PERSIST_TWO_MMA 1
+#define DPS_PERSIST_TWO_MMA 2   // 0: never; 1: grouped launches only; 2: every tile with two row blocks
 #endif
 __host__ __device__ constexpr bool persist_two_mma(bool grouped, int rb) {
-    return DPS_PERSIST_TWO_MMA != 0 && persist_x_slots(grouped) > 0 && rb == 2;
+    return rb == 2 && (DPS_PERSIST_TWO_MMA == 2 || (DPS_PERSIST_TWO_MMA == 1 && persist_x_slots(grouped) > 0));
 }
 __host__ __device__ constexpr int persist_threads(bool full, int tn, bool grouped, int rb) {
     return cta_threads(full, tn) + (persist_two_mma(grouped, rb) ? 32 : 0);
@@ -1019,7 +1022,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         for (int s = 0; s < num_stages; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
             // the zip warps that read the stage, and the tcgen05.commit if the activations ride in it
-            mbar_init(smem_u32(&bar_empty[s]), (RB == 2 ? 8 : 4) + (kXS ? 0 : 1));
+            mbar_init(smem_u32(&bar_empty[s]), (RB == 2 ? 8 : 4) + (kXS ? 0 : kMmaWarps));
         }
         for (int a = 0; a < kMaxAStages; ++a) {
             mbar_init(smem_u32(&bar_a_full[a]), 4);
