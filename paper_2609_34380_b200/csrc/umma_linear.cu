@@ -1175,7 +1175,7 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
         // ---------------- MMA issuer (one, or one per row block) ----------------
         const int w = warp == 1 ? 0 : 1;
         int s = 0;
-        int cnt[2] = {0, 0};
+        int cnt0 = 0, cnt1 = 0;   // K blocks taken from each zip group (two scalars: an array indexed by the group lives in local memory)
         int it = 0;
         int xslot = 0;            // activation slot of the next K block (launches with activation slots)
         uint32_t xparity = 0;
@@ -1209,10 +1209,11 @@ umma_persistent_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_c
                     // RB == 2: zip group rb serves row block rb of every K block; RB == 1: group s % 2
                     const int g = RB == 2 ? rb : (s & 1);
                     const int g_slots = RB == 2 ? 2 : (kTotalSlots - g + 1) / 2;
-                    const int turn = g_slots == 2 ? (cnt[g] & 1) : 0;
+                    const int cnt_g = g ? cnt1 : cnt0;
+                    const int turn = g_slots == 2 ? (cnt_g & 1) : 0;
                     const int a = RB == 2 ? 2 * g + turn : g + 2 * turn;
-                    const uint32_t a_parity = (uint32_t)(g_slots == 2 ? (cnt[g] >> 1) : cnt[g]) & 1u;
-                    ++cnt[g];
+                    const uint32_t a_parity = (uint32_t)(g_slots == 2 ? (cnt_g >> 1) : cnt_g) & 1u;
+                    if (g) ++cnt1; else ++cnt0;
                     ok = mbar_wait(smem_u32(&bar_a_full[a]), a_parity);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
