@@ -9,12 +9,14 @@
 // is "swapped": D[row][token] = sum_k W[row][k] * x[token][k], so that even a handful of decode
 // tokens fills the 128-lane datapath with weight rows and every weight byte is fetched once.
 //
-// Roles (10 warps):
+// Roles (10 warps; 11 in persistent tiles of two row blocks):
 //   warp 0     TMA producer: P tile (128 rows x 128 or 64 bytes), R tile (full mode), x tile (TN rows
 //              of 64-element swizzle atoms) into a ring of shared-memory stages, completion
-//              counted on mbarriers.  32-token tiles keep x in three slots of their own.
+//              counted on mbarriers.  Decode tiles with a K split and grouped persistent tiles keep x
+//              in slots of their own, a second stream with its own barriers (see x_slots below).
 //   warp 1     allocates tensor memory; one elected lane issues tcgen05.mma (A from TMEM, B from
-//              smem) and commits stage-release barriers.
+//              smem) and commits stage-release barriers.  Persistent tiles of two row blocks have a
+//              second issuer (warp 10), one per row block.
 //   warps 2-9  two groups of four "zip" warps; a warp owns 32 TMEM lanes = 32 weight rows.  Per K
 //              block a thread reads its row's plane bytes (swizzled, conflict-free), rebuilds the
 //              FP16 words in registers (byte permutes; hardware FP8 conversion for E4M3 fast mode)
