@@ -1832,7 +1832,7 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
     // Prefill: in full mode the zip warps (two planes to read, more bit work) are the bottleneck,
     // and a 256-token tile halves their work per FLOP (one CTA per SM, each rebuilt weight block
     // feeds twice the columns); in fast mode two co-resident 128-token CTAs with deeper rings win.
-    // DPS_FORCE_TN=128|256 overrides (tuning knob).
+    // DPS_FORCE_TN=64|128|256 overrides (tuning knob).
     static const int tn_forced = [] {
         const char* e = getenv("DPS_FORCE_TN");
         return e ? atoi(e) : 0;
@@ -1841,6 +1841,15 @@ cudaError_t launch_enc(const void* x, const uint8_t* p, const uint8_t* r, void* 
         const char* e = getenv("DPS_DENSE_RB");
         return e ? atoi(e) : 0;
     }();
+    // 65-128 tokens on matrices of moderate size: two 64-token tiles per 128 weight rows (the decode tiles with
+    // their separate plane and activation streams) instead of one 128-token tile whose K is split over a
+    // cluster and summed by remote loads.  Every weight is then streamed out of L2 and rebuilt twice, which
+    // full mode and large matrices do not forgive.  Measured at 96 and 128 tokens: Llama-7B QKV / o / down in
+    // fast mode 24.6 / 12.3-13.3 / 23.6 us against 31.7-33.8 / 19.5-20.5 / 25.6-26.6, o in full mode 17.4 against
+    // 21.5-22.6; gate/up (90 M weights) 8 % slower in fast and 30 % in full mode, hidden-8192 layers 3-50 % slower
+    // except o in fast mode (-8 %).  DPS_FORCE_TN=64|128 overrides.
+    const bool two_by_64 = tn_forced ? tn_forced == 64 : N * K <= ((int64_t)1 << (FULL ? 25 : 26));
+    if (M <= 128 && two_by_64) return launch_tn<ENC, FULL, 64>(x, p, r, y, M, N, K, status, stream);
     // Fast mode with more such tiles than SMs (the persistent kernel then walks them): 256 weight rows per CTA share
     // each 128-token activation tile, which halves the activation bytes pulled out of L2 per
     // FLOP (measured +2-8 % at 2048-8192 tokens; with fewer tiles the SMs run dry, and in full
