@@ -101,3 +101,45 @@ def test_chain_inside_a_cuda_graph(mode):
             for layer, (a, b) in enumerate(zip(bufs, drained)):
                 assert torch.equal(a.view(torch.int16), b.view(torch.int16)), f"layer {layer}"
     assert dps.dps_stream_status() == dps.DPS_OK
+
+
+@gpu
+@pytest.mark.parametrize("mode", [dps.DPS_MODE_FAST, dps.DPS_MODE_FULL])
+@pytest.mark.parametrize("T", [24, 160])
+def test_grouped_chain_equals_drained_chain(T, mode):
+    # a gate/up-style call (token map) followed by down-style calls (rows are their own tokens), every output
+    # the next input, with one workspace shared by all calls as a serving loop would
+    E, N = 4, 1024
+    K = N
+    ps, rs, encs = [], [], []
+    for e in range(E):
+        w = workloads.weights(N, K, 7500 + e, device=DEV)
+        w = (w.float() * (1.0 / (w.float().std().item() * K ** 0.5))).to(torch.float16)
+        p, r, enc, _, _ = split_both(w, dps.DPS_ENC_AUTO, DEV)
+        ps.append(p), rs.append(r), encs.append(enc)
+    p, r = torch.stack(ps), torch.stack(rs)
+    tor, eor = workloads.top2_routing(T, E, 7600 + T)
+    tor_d, eor_d = torch.from_numpy(tor).to(DEV), torch.from_numpy(eor).to(DEV)
+    A = eor.size
+    x0 = workloads.activations(T, K, 7700 + T, device=DEV)
+    ws = torch.empty(dps.dps_moe_workspace_bytes(A, E, K), dtype=torch.uint8, device=DEV)
+
+    def chain(drain):
+        outs = []
+        x, tmap = x0, tor_d
+        for _ in range(6):
+            y = torch.empty((A, N), dtype=torch.float16, device=DEV)
+            dps.dps_moe_linear(mode, encs, x, tmap, eor_d, p, r if mode else None, y, ws)
+            if drain:
+                torch.cuda.synchronize()
+            outs.append(y)
+            x, tmap = y, None
+        torch.cuda.synchronize()
+        return outs
+
+    drained = chain(True)
+    for attempt in range(3):
+        for layer, (a, b) in enumerate(zip(chain(False), drained)):
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16)), f"layer {layer}, attempt {attempt}"
+    assert torch.isfinite(drained[-1].float()).all()
+    assert dps.dps_stream_status() == dps.DPS_OK
