@@ -1440,12 +1440,14 @@ int forced_split() {
 // K split for a launch of `tiles` output tiles.  capacity[s] = CTAs that can be resident at once
 // when launched as clusters of s (clusters must fit inside one GPC, so this is not a multiple of
 // the SM count).  Measured on B200: a second wave costs more than it buys, so take the largest
-// factor (<= 8, a portable cluster) whose CTAs are all resident at once, keeping at least 4 K
-// blocks per CTA.
-int choose_split(int64_t tiles, int total_kb, const int* capacity) {
+// factor (<= 8, a portable cluster) whose CTAs are all resident at once, keeping at least min_kb K
+// blocks per CTA: 4 in fast mode, 5 in full mode (4096 x 4096 at 32-64 tokens in full mode: 6 CTAs per
+// tile are 3-5 % faster than 8 with 4 blocks each, alone and inside the decode graphs; in fast mode they
+// are as fast alone and 4 % slower inside the graphs).
+int choose_split(int64_t tiles, int total_kb, const int* capacity, int min_kb) {
     int best = 1;
     for (int s = 2; s <= kMaxSplit; ++s) {
-        if (total_kb / s < 4) break;
+        if (total_kb / s < min_kb) break;
         if (tiles * s <= capacity[s]) best = s;
     }
     return best;
@@ -1688,7 +1690,7 @@ cudaError_t launch_tn(const void* x, const uint8_t* p, const uint8_t* r, void* y
     const int64_t row_tiles = (N + kTileRows - 1) / kTileRows, tok_tiles = (M + TN - 1) / TN;
     const int total_kb = (int)((K + kBlockK - 1) / kBlockK);
     int split = forced_split();
-    if (split <= 0) split = choose_split(row_tiles * tok_tiles, total_kb, capacity);
+    if (split <= 0) split = choose_split(row_tiles * tok_tiles, total_kb, capacity, FULL ? 5 : 4);
     if (deep) split = 1;
     (void)tiles_total;
     if (split > total_kb) split = total_kb;
