@@ -279,12 +279,17 @@ cudaError_t launch_one(const __half* x, const uint8_t* p, const uint8_t* r, __ha
     cfg.numAttrs = 1;
     // DPS_STREAM_PREFETCH=<steps> overrides how many 2 KB column steps of its row block a CTA asks
     // L2 for before it waits for the preceding kernel (0 = none), DPS_STREAM_PREFETCH_CTAS how many
-    // CTAs of the grid do so.  Measured on Llama-7B shapes: one step by the first wave of CTAs gains
-    // 1-10 %; whole row blocks, or every CTA of a grid of several waves, lose.
-    static const int prefetch_steps = [] {
+    // CTAs of the grid do so.  Measured on Llama-7B shapes, every launch timed in a loop of its own: one step
+    // by the first wave of CTAs gains 1-10 %; whole row blocks, or every CTA of a grid of several waves, lose.
+    // Inside a decoder's chain of launches (graphs of 128 launches, the four Llama-7B linears in turn) the
+    // picture differs by mode: fast mode keeps 2 % of that gain at 8 tokens, full mode LOSES 4-6 % to it (1 and
+    // 8 tokens: 0.85 / 0.83 of the copy bandwidth with the prefetch, 0.90 / 0.87 without -- the requests compete
+    // with the tail of the launch in front, which in full mode streams twice as long).  So: fast mode only.
+    static const int prefetch_forced = [] {
         const char* e = getenv("DPS_STREAM_PREFETCH");
-        return e ? atoi(e) : 1;
+        return e ? atoi(e) : -1;
     }();
+    const int prefetch_steps = prefetch_forced >= 0 ? prefetch_forced : (FULL ? 0 : 1);
     static const int prefetch_ctas = [] {
         const char* e = getenv("DPS_STREAM_PREFETCH_CTAS");
         return e ? atoi(e) : 2 * sm_count();
