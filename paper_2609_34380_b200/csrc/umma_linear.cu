@@ -125,6 +125,12 @@ __host__ __device__ constexpr int tmem_cols(bool full, int tn, int rb = 1) {
 #ifndef DPS_XSLOT_MAX_TN
 #define DPS_XSLOT_MAX_TN 32
 #endif
+// Plane loading ahead of the dependency in decode tiles (see kPre in the kernel).  Measured inside the decode
+// graphs at 32 tokens (fast / full, fraction of the copy bandwidth): nothing 0.55 / 0.60, the first ring pass
+// 0.58 / 0.67, refills too 0.59 / 0.71, with the L2 prefetch of the second pass the same.
+#ifndef DPS_PRE_DEP
+#define DPS_PRE_DEP 3
+#endif
 #ifndef DPS_XSLOTS
 #define DPS_XSLOTS 5        // fast mode
 #endif
@@ -530,11 +536,14 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
             for (int t = 0; t < kXAtoms; ++t)
                 tma_load_2d(dst + (uint32_t)(t * TN * 128), &map_x, full, k + t * 64, m0);
         };
+        // How much of that a tile with activation slots does ahead of the dependency (tuning knob): 0 nothing,
+        // 1 the first ring pass, 2 also refills of stages the zip warps hand back, 3 also the L2 prefetch.
+        constexpr int kPre = kXS ? DPS_PRE_DEP : 3;
         if (!GROUPED && elect_one()) {
-            for (int i = 0; i < first; ++i) load_planes(i, i);
+            for (int i = 0; kPre >= 1 && i < first; ++i) load_planes(i, i);
             // ... and the plane tiles of the second pass are pulled into L2 meanwhile.
             // (A rolling L2 prefetch further ahead during the main loop was measured slower.)
-            const int ahead = num_kb < 2 * num_stages ? num_kb : 2 * num_stages;
+            const int ahead = kPre >= 3 ? (num_kb < 2 * num_stages ? num_kb : 2 * num_stages) : 0;
             for (int i = first; i < ahead; ++i) {
                 const int k = (rank + i * split) * kBlockK;
                 tma_prefetch_l2_2d(&map_p, k, plane_row0);
@@ -580,15 +589,17 @@ umma_linear_kernel(const __grid_constant__ CUtensorMap map_p, const __grid_const
         // whichever barrier comes next in each stream, so that neither stream waits for the other's consumer;
         // the clock is read once in a while to keep the wait bounded.
         if (kXS) {
-            int ip = first, ix = 0;                                     // next K block of each stream
-            int sp = first == num_stages ? 0 : first, sx = 0;           // its stage / slot
-            uint32_t php = 0u, phx = 0u;                                // parity of the "free" phase awaited there
+            int ip = kPre >= 1 ? first : 0, ix = 0;                     // next K block of each stream
+            int sp = ip == num_stages ? 0 : ip, sx = 0;                 // its stage / slot
+            // parity of the "free" phase awaited there (a fresh barrier passes a wait for the phase before its first)
+            uint32_t php = ip == num_stages ? 0u : 1u, phx = 0u;
             bool dep = false;                                           // the preceding kernel's output may be read
             uint32_t idle = 0;
             unsigned long long t0 = 0;
             while ((ip < num_kb || ix < num_kb) && ok) {
                 bool progress = false;
-                if (ip < num_kb && __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_empty[sp]), php))) {
+                if (ip < num_kb && (kPre >= 2 || dep) &&
+                    __any_sync(0xFFFFFFFFu, mbar_test_wait(smem_u32(&bar_empty[sp]), php))) {
                     DPS_STAMP(0, ip);
                     if (elect_one()) load_planes(ip, sp);
                     __syncwarp();
